@@ -1,0 +1,220 @@
+/*
+ * flashbev_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, fp64 CPU statement of the Sampling-VT operator (paper Eq. 1,
+ * Sec. 3.1) evaluated in the loop order of the fused algorithm (Algorithm 2):
+ * for every BEV cell, for every height bin z, for every camera n: voxel centre
+ * -> projection -> validity mask M_n -> bilinear sample f_n -> per-z camera
+ * reduction -> sum over z.  Nothing here is blocked, fused, vectorised or
+ * reordered beyond that; the only concession to run time is an OpenMP
+ * "parallel for" over BEV cells, which Sec. 3.2.2 states are independent.
+ *
+ * Only the tests, the smoke check and the bench's CPU-baseline leg may call
+ * this file.  It shares no source, header, table or helper with the CUDA
+ * library and neither includes the other.
+ *
+ * Conventions (each one is a reading of the paper or of the operator's
+ * interface statement; they are listed with their justification in the design
+ * notes):
+ *   - voxel centres are BIN centres on all three axes:
+ *       x_w = x_min + (ix + 1/2) (x_max - x_min) / X        (Sec. 4.1: [-50,50] m
+ *       at 0.5 m <-> X = 200, [-5,5] m at 1.25 m <-> Z = 8: bins, not linspace)
+ *   - the 4x4 matrix maps homogeneous metres to (u d, v d, d) in full-resolution
+ *     image pixels; only rows 0..2 are read
+ *   - M_n = 1 iff d > 0.1 and the sample lies strictly inside the feature map
+ *     under grid_sample(align_corners=False) conventions:
+ *       fx = u Wf / Wimg - 1/2,  fy = v Hf / Himg - 1/2,
+ *       -1/2 < fx < Wf - 1/2,   -1/2 < fy < Hf - 1/2
+ *   - f_n is bilinear interpolation with zero padding: a tap outside
+ *     [0,Wf-1] x [0,Hf-1] contributes 0, the sample still counts in den_z
+ *   - reduce = 0 (SUM):                out = sum_z sum_n M f
+ *     reduce = 1 (MEAN_OVER_VALID):    out = (sum_z sum_n M f) / max(1, sum_z sum_n M)
+ *     reduce = 2 (CAMERA_MEAN_Z_SUM):  out = sum_z [ sum_n M f / max(1, sum_n M) ]   (Eq. 1)
+ *
+ * Parity pins (tests/, CPU only): constant and affine feature maps (closed
+ * forms), camera permutation, linearity, z-split additivity, grid-subset
+ * invariance, a hand-computed one-sample case, an orthographic special case
+ * against a library bilinear resampler, the Alg. 1 (tensorised) order written
+ * independently in numpy, and the identities that tie the three reduce modes
+ * together.  Which normalisation the interface's "mean_over_valid" means is a
+ * reading, not something the paper fixes: for reduce = 1 parity is pinned to
+ * that reading only ("parity unpinned" with respect to the paper).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_DEPTH_MIN 0.1    /* metres; interface statement: camera depth > 0.1 m */
+#define ORACLE_BORDER_EPS 1e-3  /* feature px (image borders) / metres (depth plane) */
+
+int flashbev_oracle_version(void) { return 1; }
+
+int flashbev_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/*
+ * features  : host, float32 [B][N][Hf][Wf][C]  (bf16 workloads pass the bf16-rounded
+ *             values, which are exact in float32; everything is widened to double)
+ * lidar2img : host, float32 [B][N][4][4] row-major
+ * out       : host, double  [B][X][Y][C]
+ * count     : host, int32   [B][X][Y]   sum over z,n of M_n                 (may be NULL)
+ * flagged   : host, int32   [B][X][Y]   samples within ORACLE_BORDER_EPS of a
+ *                                        validity border                    (may be NULL)
+ * sumw      : host, double  [B][X][Y]   sum over valid samples of the in-bounds
+ *                                        bilinear weight mass               (may be NULL)
+ * interior  : host, uint8   [B][X][Y]   1 iff every valid sample has all four taps
+ *                                        inside the map                     (may be NULL)
+ * nzbins    : host, int32   [B][X][Y]   number of z bins with den_z > 0     (may be NULL)
+ * nthreads  : OpenMP threads over cells (<= 0: library default)
+ * returns 0, or -1 on a bad argument, -2 if out of memory.
+ */
+int flashbev_oracle_sampling_vt(const float *features, const float *lidar2img,
+                                int B, int N, int C, int Hf, int Wf, int Himg, int Wimg,
+                                double x_min, double x_max, double y_min, double y_max,
+                                double z_min, double z_max, int X, int Y, int Z, int reduce,
+                                double *out, int32_t *count, int32_t *flagged, double *sumw,
+                                uint8_t *interior, int32_t *nzbins, int nthreads)
+{
+    if (!features || !lidar2img || !out) return -1;
+    if (B <= 0 || N <= 0 || C <= 0 || Hf <= 0 || Wf <= 0 || Himg <= 0 || Wimg <= 0) return -1;
+    if (X <= 0 || Y <= 0 || Z <= 0 || reduce < 0 || reduce > 2) return -1;
+    if (!(x_max > x_min) || !(y_max > y_min) || !(z_max > z_min)) return -1;
+
+    const double sx = (double)Wf / (double)Wimg; /* image px -> feature px */
+    const double sy = (double)Hf / (double)Himg;
+    const long long cells = (long long)B * X * Y;
+    int oom = 0;
+#ifdef _OPENMP
+    if (nthreads <= 0) nthreads = omp_get_max_threads();
+#else
+    nthreads = 1;
+#endif
+
+#pragma omp parallel num_threads(nthreads)
+    {
+        double *acc = (double *)malloc(sizeof(double) * (size_t)C);
+        double *num = (double *)malloc(sizeof(double) * (size_t)C);
+        if (!acc || !num) {
+#pragma omp atomic write
+            oom = 1;
+        }
+#pragma omp barrier
+        if (!oom) {
+#pragma omp for schedule(dynamic, 16)
+            for (long long cell = 0; cell < cells; ++cell) {
+                const int b = (int)(cell / ((long long)X * Y));
+                const int ix = (int)((cell / Y) % X);
+                const int iy = (int)(cell % Y);
+                /* voxel centre (Alg. 2 "compute voxel center"): bin centres */
+                const double xw = x_min + ((double)ix + 0.5) * (x_max - x_min) / (double)X;
+                const double yw = y_min + ((double)iy + 0.5) * (y_max - y_min) / (double)Y;
+
+                for (int c = 0; c < C; ++c) acc[c] = 0.0;
+                int32_t cnt = 0, flg = 0, nzb = 0;
+                double sw = 0.0;
+                int inter = 1;
+
+                for (int k = 0; k < Z; ++k) { /* z outer, n inner: Alg. 2 */
+                    const double zw = z_min + ((double)k + 0.5) * (z_max - z_min) / (double)Z;
+                    for (int c = 0; c < C; ++c) num[c] = 0.0;
+                    int den = 0;
+
+                    for (int n = 0; n < N; ++n) {
+                        const float *M = lidar2img + ((size_t)b * N + n) * 16;
+                        /* projection: rows 0..2 of M times (x_w, y_w, z_w, 1) */
+                        const double p0 = (double)M[0] * xw + (double)M[1] * yw + (double)M[2] * zw + (double)M[3];
+                        const double p1 = (double)M[4] * xw + (double)M[5] * yw + (double)M[6] * zw + (double)M[7];
+                        const double d = (double)M[8] * xw + (double)M[9] * yw + (double)M[10] * zw + (double)M[11];
+
+                        /* M_n, first half: positive depth (also rejects NaN) */
+                        const int in_front = (d > ORACLE_DEPTH_MIN);
+                        if (!in_front && !(d > ORACLE_DEPTH_MIN - ORACLE_BORDER_EPS)) continue;
+                        /* here d > 0.099, so the perspective division is well defined */
+
+                        const double u = p0 / d; /* image pixels */
+                        const double v = p1 / d;
+                        const double fx = u * sx - 0.5; /* feature pixels, align_corners=False */
+                        const double fy = v * sy - 0.5;
+
+                        /* signed distances to the four image borders (feature px) and to
+                           the depth plane (m); the smallest one decides validity */
+                        const double mx0 = fx + 0.5, mx1 = ((double)Wf - 0.5) - fx;
+                        const double my0 = fy + 0.5, my1 = ((double)Hf - 0.5) - fy;
+                        const double md = d - ORACLE_DEPTH_MIN;
+                        const int in_img = (mx0 > 0.0) && (mx1 > 0.0) && (my0 > 0.0) && (my1 > 0.0);
+                        if (isfinite(fx) && isfinite(fy)) {
+                            double m = md;
+                            if (mx0 < m) m = mx0;
+                            if (mx1 < m) m = mx1;
+                            if (my0 < m) m = my0;
+                            if (my1 < m) m = my1;
+                            /* border sample: its validity may legitimately differ between
+                               two correct implementations; reported, excluded from parity */
+                            if (fabs(m) < ORACLE_BORDER_EPS) flg += 1;
+                        }
+                        if (!in_front || !in_img) continue; /* M_n = 0 */
+
+                        /* bilinear sample f_n with zero padding */
+                        const double x0f = floor(fx), y0f = floor(fy);
+                        const int x0 = (int)x0f, y0 = (int)y0f;
+                        const double tx = fx - x0f, ty = fy - y0f;
+                        const float *Fn = features + ((size_t)b * N + n) * (size_t)Hf * Wf * C;
+                        double wsum = 0.0;
+                        int all_in = 1;
+                        for (int dy = 0; dy < 2; ++dy) {
+                            for (int dx = 0; dx < 2; ++dx) {
+                                const int xi = x0 + dx, yi = y0 + dy;
+                                const double w = (dx ? tx : 1.0 - tx) * (dy ? ty : 1.0 - ty);
+                                if (xi < 0 || xi > Wf - 1 || yi < 0 || yi > Hf - 1) {
+                                    all_in = 0;
+                                    continue;
+                                }
+                                const float *t = Fn + ((size_t)yi * Wf + xi) * C;
+                                for (int c = 0; c < C; ++c) num[c] += w * (double)t[c];
+                                wsum += w;
+                            }
+                        }
+                        den += 1;
+                        sw += wsum;
+                        if (!all_in) inter = 0;
+                    }
+
+                    cnt += den;
+                    if (den > 0) nzb += 1;
+                    if (reduce == 2) {
+                        const double dz = (double)(den > 1 ? den : 1); /* g_z = num_z / max(1, den_z) */
+                        for (int c = 0; c < C; ++c) acc[c] += num[c] / dz;
+                    } else {
+                        for (int c = 0; c < C; ++c) acc[c] += num[c];
+                    }
+                }
+
+                double *o = out + (size_t)cell * C;
+                if (reduce == 1) {
+                    const double dn = (double)(cnt > 1 ? cnt : 1);
+                    for (int c = 0; c < C; ++c) o[c] = acc[c] / dn;
+                } else {
+                    for (int c = 0; c < C; ++c) o[c] = acc[c];
+                }
+                if (count) count[cell] = cnt;
+                if (flagged) flagged[cell] = flg;
+                if (sumw) sumw[cell] = sw;
+                if (interior) interior[cell] = (uint8_t)inter;
+                if (nzbins) nzbins[cell] = nzb;
+            }
+        }
+        free(acc);
+        free(num);
+    }
+    return oom ? -2 : 0;
+}

@@ -1,0 +1,95 @@
+"""ctypes front end of the fp64 CPU oracle -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+
+Builds ``flashbev_oracle.c`` with gcc on first use and exposes ``sampling_vt``.
+Only the tests, the smoke check and the bench's CPU-baseline leg may import this
+module; it imports nothing from the CUDA package and the CUDA package imports
+nothing from here.
+
+The arithmetic lives entirely in the C file (paper Eq. 1 / Algorithm 2); this
+module only marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "flashbev_oracle.c")
+_LIB = os.path.join(_HERE, "libflashbev_oracle.so")
+
+REDUCE_SUM = 0
+REDUCE_MEAN_OVER_VALID = 1
+REDUCE_CAMERA_MEAN_Z_SUM = 2  # paper Eq. 1
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (plain gcc, OpenMP over cells, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-std=c99", "-O2", "-fopenmp", "-ffp-contract=off", "-Wall", "-Wextra",
+               "-shared", "-fPIC", _SRC, "-o", _LIB, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        d, i, p = ctypes.c_double, ctypes.c_int, ctypes.c_void_p
+        lib.flashbev_oracle_sampling_vt.restype = i
+        lib.flashbev_oracle_sampling_vt.argtypes = (
+            [p, p] + [i] * 7 + [d] * 6 + [i] * 4 + [p] * 6 + [i])
+        lib.flashbev_oracle_max_threads.restype = i
+        _lib = lib
+    return _lib
+
+
+def max_threads() -> int:
+    return int(_load().flashbev_oracle_max_threads())
+
+
+@dataclass
+class OracleResult:
+    out: np.ndarray        # float64 [B, X, Y, C]
+    count: np.ndarray      # int32   [B, X, Y]  valid samples per cell
+    flagged: np.ndarray    # int32   [B, X, Y]  border samples per cell
+    sumw: np.ndarray       # float64 [B, X, Y]  in-bounds bilinear weight mass
+    interior: np.ndarray   # bool    [B, X, Y]  all taps of all valid samples in bounds
+    nzbins: np.ndarray     # int32   [B, X, Y]  height bins seen by at least one camera
+
+
+def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM, threads=0) -> OracleResult:
+    """Run the oracle.
+
+    features : float32 array [B, N, Hf, Wf, C] (bf16 workloads: bf16-rounded values)
+    lidar2img: float32 array [B, N, 4, 4]
+    img_hw   : (Himg, Wimg)
+    bev_range: (x_min, x_max, y_min, y_max, z_min, z_max) in metres
+    grid     : (X, Y, Z)
+    """
+    f = np.ascontiguousarray(features, dtype=np.float32)
+    m = np.ascontiguousarray(lidar2img, dtype=np.float32)
+    if f.ndim != 5 or m.shape != (f.shape[0], f.shape[1], 4, 4):
+        raise ValueError("features must be [B,N,Hf,Wf,C] and lidar2img [B,N,4,4]")
+    B, N, Hf, Wf, C = f.shape
+    X, Y, Z = (int(v) for v in grid)
+    out = np.empty((B, X, Y, C), np.float64)
+    count = np.empty((B, X, Y), np.int32)
+    flagged = np.empty((B, X, Y), np.int32)
+    sumw = np.empty((B, X, Y), np.float64)
+    interior = np.empty((B, X, Y), np.uint8)
+    nzbins = np.empty((B, X, Y), np.int32)
+    rc = _load().flashbev_oracle_sampling_vt(
+        f.ctypes.data, m.ctypes.data, B, N, C, Hf, Wf, int(img_hw[0]), int(img_hw[1]),
+        *(float(v) for v in bev_range), X, Y, Z, int(reduce),
+        out.ctypes.data, count.ctypes.data, flagged.ctypes.data, sumw.ctypes.data,
+        interior.ctypes.data, nzbins.ctypes.data, int(threads))
+    if rc != 0:
+        raise ValueError(f"flashbev_oracle_sampling_vt rejected its arguments (status {rc})")
+    return OracleResult(out, count, flagged, sumw, interior.astype(bool), nzbins)

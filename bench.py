@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the fused Sampling-VT operator on B200.
+
+A *step* is one pass of the whole operator (stage matrices -> project -> validity -> bilinear
+weights -> per-z normalisation -> gather/accumulate -> store) over one batch of FRAMES
+independent synthetic frames of the chosen workload, each frame one call of
+``flashbev_sampling_vt`` through the C ABI on its own device-resident inputs.  The frames of a
+step together exceed the L2 cache several times over, so every launch starts L2-cold without an
+explicit flush.  The launches of a step are replayed from a CUDA graph so that the number is the
+GPU's, not the Python launch loop's (``--no-graph`` times direct launches instead).
+
+Prints ONE JSON line.  ``value`` is whole-job sample-channels/s (all B*N*X*Y*Z*C candidate
+sample-channels of every frame on every rank / device time, max over ranks).
+
+``--impl reference`` times the fp64 CPU oracle (a deliberately plain program) on the host cores
+for the same workload and metric.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_10071_b200 import workloads as wl  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "fused_sampling_vt_throughput"
+UNIT = "sample-channels/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def frames_for(w: wl.Workload, min_bytes: int) -> int:
+    return max(4, -(-min_bytes // w.unique_bytes))
+
+
+def oracle_throughput(w: wl.Workload, seconds_budget: float, max_frames: int):
+    """Time the oracle as it stands on the host cores over whole frames of the workload."""
+    from oracle import flashbev_oracle as orc
+    orc.build()
+    inp = wl.make_inputs(w)
+    t0 = time.perf_counter()
+    frames = 0
+    while frames < max_frames and (frames == 0 or time.perf_counter() - t0 < seconds_budget):
+        orc.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, w.reduce)
+        frames += 1
+    dt = time.perf_counter() - t0
+    return {"value": frames * w.sample_channels / dt, "unit": UNIT, "cores": orc.max_threads(), "kind": "oracle",
+            "sample": f"{frames} whole frame(s) of the '{w.name}' workload, {dt / frames * 1e3:.1f} ms each",
+            "ms_per_frame": dt / frames * 1e3}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import flashbev_oracle as orc
+    orc.build()
+    inp = wl.make_inputs(w)
+    frames_per_step = 1
+    for _ in range(args.warmup):
+        orc.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, w.reduce)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, w.reduce)
+    dt = time.perf_counter() - t0
+    value = args.steps * frames_per_step * w.sample_channels / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "frames_per_step": frames_per_step, "note": "fp64 CPU oracle on the host cores"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.max_threads(), "kind": "oracle",
+                         "sample": f"{frames_per_step} whole frame of '{w.name}' per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+class DeviceFrames:
+    """FRAMES independent frames of one workload, resident on the device, with their parameter structs."""
+
+    def __init__(self, w, frames, device, rank, kernel=0, tune=(0, 0, 0, 0)):
+        import torch
+        from paper_2607_10071_b200 import binding as fb
+        self.w, self.frames = w, frames
+        X, Y, Z = w.grid
+        self.feats, self.mats, self.outs, self.params = [], [], [], []
+        base = wl.make_inputs(w, stream=1000 * rank)
+        g = torch.Generator(device="cpu").manual_seed(2607_10071 + rank)
+        for i in range(frames):
+            if i == 0:
+                f32 = torch.from_numpy(base.features)
+            else:  # same shape and distribution, different values (standard normal, seeded)
+                f32 = torch.randn(base.features.shape, generator=g, dtype=torch.float32)
+            f = f32.to(device)
+            if w.dtype == "bf16":
+                f = f.to(torch.bfloat16)
+            self.feats.append(f.contiguous())
+            self.mats.append(torch.from_numpy(base.lidar2img).to(device))
+            self.outs.append(torch.empty((w.B, X, Y, w.C), dtype=torch.float32, device=device))
+            self.params.append(fb.make_params(
+                self.feats[-1].data_ptr(), fb.BF16 if w.dtype == "bf16" else fb.F32, self.mats[-1].data_ptr(),
+                w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid, w.reduce, self.outs[-1].data_ptr(),
+                None, kernel, tune))
+        self.fb = fb
+
+    def launch_all(self, stream_ptr):
+        n = 0
+        for p in self.params:
+            self.fb.flashbev_sampling_vt(p, stream_ptr)
+            n += self.fb.flashbev_last_launch_count()
+        return n
+
+
+def time_steps(torch, step_fn, steps, warmup, dist_barrier):
+    """Device time of `steps` steps: per-step CUDA events on the current stream."""
+    for _ in range(warmup):
+        step_fn()
+    torch.cuda.synchronize()
+    dist_barrier()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t_all0, t_all1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_all0.record()
+    for a, b in evs:
+        a.record()
+        step_fn()
+        b.record()
+    t_all1.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    torch.cuda.synchronize()
+    per = [a.elapsed_time(b) for a, b in evs]
+    return t_all0.elapsed_time(t_all1), per
+
+
+def measure_workload(torch, w, args, device, rank, dist_barrier, steps, warmup, kernel=0, tune=(0, 0, 0, 0)):
+    frames = args.frames or frames_for(w, 3 * L2_BYTES)
+    df = DeviceFrames(w, frames, device, rank, kernel, tune)
+    stream = torch.cuda.Stream(device)
+    launches_per_step = frames
+    with torch.cuda.stream(stream):
+        sp = stream.cuda_stream
+        df.launch_all(sp)  # first call: module load
+        torch.cuda.synchronize()
+        if args.no_graph:
+            def step_fn():
+                df.launch_all(sp)
+        else:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                df.launch_all(torch.cuda.current_stream().cuda_stream)
+
+            def step_fn():
+                graph.replay()
+        total_ms, per = time_steps(torch, step_fn, steps, warmup, dist_barrier)
+    kname = df.fb.flashbev_last_kernel_name()
+    return {"frames": frames, "total_ms": total_ms, "per_step_ms": per, "launches_per_step": launches_per_step,
+            "kernel": kname, "df": df}
+
+
+def measure_e2e(torch, w, args, device, steps, warmup, dist_barrier):
+    """Same metric through flashbev_sampling_vt_host: pinned host inputs, host output, copies timed."""
+    from paper_2607_10071_b200 import binding as fb
+    frames = max(2, min(args.frames or frames_for(w, 3 * L2_BYTES), 8))
+    X, Y, Z = w.grid
+    inp = wl.make_inputs(w)
+    if w.dtype == "bf16":
+        hf = torch.from_numpy(inp.features_bf16.view(np.int16)).pin_memory()
+    else:
+        hf = torch.from_numpy(inp.features).pin_memory()
+    hm = torch.from_numpy(inp.lidar2img).pin_memory()
+    houts = [torch.empty((w.B, X, Y, w.C), dtype=torch.float32).pin_memory() for _ in range(frames)]
+    ps = [fb.make_params(hf.data_ptr(), fb.BF16 if w.dtype == "bf16" else fb.F32, hm.data_ptr(), w.B, w.N, w.C,
+                         w.feat_hw, w.img_hw, w.bev_range, w.grid, w.reduce, ho.data_ptr()) for ho in houts]
+    need = fb.flashbev_host_staging_bytes(ps[0])
+    stagings = [torch.empty(need, dtype=torch.uint8, device=device) for _ in range(frames)]
+    stream = torch.cuda.Stream(device)
+    sp = stream.cuda_stream
+
+    def step_fn():
+        for p, st in zip(ps, stagings):
+            fb.flashbev_sampling_vt_host(p, st.data_ptr(), need, sp)
+
+    with torch.cuda.stream(stream):
+        total_ms, _ = time_steps(torch, step_fn, steps, warmup, dist_barrier)
+    return {"value_per_rank": steps * frames * w.sample_channels / (total_ms * 1e-3), "frames": frames,
+            "h2d": frames * (w.feature_bytes + w.matrix_bytes), "d2h": frames * w.output_bytes, "total_ms": total_ms}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="representative", choices=list(wl.WORKLOADS))
+    ap.add_argument("--frames", type=int, default=0, help="frames per step (0: enough to exceed 3x L2)")
+    ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a CUDA graph replay")
+    ap.add_argument("--no-table", action="store_true", help="skip the per-configuration table")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 per-output, 2 tiled")
+    ap.add_argument("--tune", type=str, default="0,0,0,0")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = wl.get(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2607_10071_b200 import binding as fb
+    from paper_2607_10071_b200 import build as fbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the operator has no CPU path")
+    if rank == 0 and fbuild.needs_build():
+        fbuild.build()
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+        def barrier():
+            dist.barrier()
+    else:
+        def barrier():
+            pass
+    barrier()
+    fb.lib()
+    tune = tuple(int(t) for t in args.tune.split(","))
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    m = measure_workload(torch, w, args, device, rank, barrier, args.steps, args.warmup, args.kernel, tune)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # max over ranks of the device time of the K steps
+    t = torch.tensor([m["total_ms"]], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    frames = m["frames"]
+    value = world * args.steps * frames * w.sample_channels / (total_ms * 1e-3)
+    launch_ms = statistics.mean(m["per_step_ms"]) / frames  # average duration of one launch (one frame)
+
+    # peak memory of one call: nothing may be allocated
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    torch.cuda.reset_peak_memory_stats()
+    a0 = torch.cuda.max_memory_allocated()
+    fb.flashbev_sampling_vt(m["df"].params[0], torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    workspace = (torch.cuda.max_memory_allocated() - a0) + max(0, free0 - torch.cuda.mem_get_info()[0])
+
+    e2e = measure_e2e(torch, w, args, device, max(3, args.steps // 4), 3, barrier)
+    te = torch.tensor([e2e["total_ms"]], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * max(3, args.steps // 4) * e2e["frames"] * w.sample_channels / (float(te.item()) * 1e-3)
+
+    table = {}
+    if not args.no_table and world == 1:
+        for name in wl.CONFIG_ORDER:
+            wi = wl.get(name)
+            mi = measure_workload(torch, wi, args, device, rank, barrier, max(3, args.steps // 4), 3)
+            mi.pop("df")
+            lat = statistics.mean(mi["per_step_ms"]) / mi["frames"]
+            peak, _ = measured_peaks()
+            table[name] = {"latency_ms": round(lat, 5), "sample_channels_per_s": wi.sample_channels / (lat * 1e-3),
+                           "hbm_roofline_frac_of_measured": wi.unique_bytes / (lat * 1e-3) / 1e9 / peak,
+                           "hbm_roofline_frac_of_8TBs": wi.unique_bytes / (lat * 1e-3) / 1e9 / 8000.0,
+                           "unique_mb": round(wi.unique_bytes / 1e6, 3), "output_mb": round(wi.output_bytes / 1e6, 3),
+                           "kernel": mi["kernel"], "frames_per_step": mi["frames"], "reduce": wi.reduce}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    achieved = w.unique_bytes / (launch_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.dtype == "f32" else "bf16 features, f32 accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "N": w.N, "C": w.C, "feat_hw": list(w.feat_hw), "img_hw": list(w.img_hw),
+                   "grid": list(w.grid), "bev_range": list(w.bev_range), "reduce": w.reduce, "frames_per_step": frames,
+                   "l2": "inputs of a step total %.0f MB (> 3x the 126 MB L2), no flush" % (frames * w.unique_bytes / 1e6),
+                   "launch": "direct" if args.no_graph else "cuda graph replay of the step's launches",
+                   "kernel": m["kernel"]},
+        "latency_ms": launch_ms,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": w.unique_bytes,
+                     "frac_of_8TBs_nominal": achieved / 8000.0},
+        "peak_mb": {"workspace_allocated_by_call": workspace / 1e6, "output": w.output_bytes / 1e6,
+                    "inputs_plus_output": w.unique_bytes / 1e6},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "frames_per_step": e2e["frames"], "api": "flashbev_sampling_vt_host (pinned host buffers)"},
+        "gpu_launches": args.steps * m["launches_per_step"],
+        "clocks": clocks,
+    }
+    if table:
+        line["configs"] = table
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = oracle_throughput(w, 12.0, 200)
+    elif world == 1:
+        line["cpu_baseline"] = None
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,145 @@
+/*
+ * flashbev.h -- C ABI of the B200 (sm_100a) fused Sampling-VT library.
+ *
+ * One operator: the exact sampling-based BEV view transformation of the FlashBEV
+ * paper, executed as a single fused gather-reduction (Sec. 3.3, Algorithm 2) so
+ * that only the B x X x Y x C output is ever written and no height-dependent
+ * intermediate exists.
+ *
+ * Plain C: pointers and sizes only.  Every pointer in `flashbev_vt_params` is a
+ * DEVICE pointer unless the entry point says otherwise.  The caller owns every
+ * buffer.  Unless an entry point says otherwise the library allocates nothing,
+ * frees nothing, keeps no pointer after return, never synchronises the device,
+ * and enqueues its work on the caller's stream.  It is re-entrant and thread safe.
+ */
+#ifndef FLASHBEV_H_
+#define FLASHBEV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FLASHBEV_VERSION 100 /* 0.1.0 */
+
+typedef enum flashbev_status {
+    FLASHBEV_OK = 0,
+    FLASHBEV_INVALID_ARG = 1,  /* null pointer, non-positive size, empty range, unknown enum, short struct */
+    FLASHBEV_UNSUPPORTED = 2,  /* a combination this version does not implement (NCHW, bf16 output, sizes
+                                  beyond the 32-bit index ranges stated below) */
+    FLASHBEV_MISALIGNED = 3,   /* `out` or `lidar2img` not 4-byte aligned, `features` not element aligned */
+    FLASHBEV_CUDA_ERROR = 4,   /* the launch (or a copy of the host entry point) failed; the CUDA error
+                                  has been consumed with cudaGetLastError */
+    FLASHBEV_TOO_SMALL = 5     /* a caller-provided staging buffer is smaller than required */
+} flashbev_status;
+
+typedef enum flashbev_dtype { FLASHBEV_F32 = 0, FLASHBEV_BF16 = 1 } flashbev_dtype;
+
+/* NHWC: features [B][N][Hf][Wf][C] and out [B][X][Y][C], C contiguous (Algorithm 2 states the
+ * output as B x X x Y x C).  NCHW is declared for ABI stability and returns FLASHBEV_UNSUPPORTED. */
+typedef enum flashbev_layout { FLASHBEV_NHWC = 0, FLASHBEV_NCHW = 1 } flashbev_layout;
+
+/*
+ * Reduction over cameras n and height bins z (M_n = validity mask, f_n = bilinear sample):
+ *   SUM               out = sum_z sum_n M_n f_n
+ *   MEAN_OVER_VALID   out = (sum_z sum_n M_n f_n) / max(1, sum_z sum_n M_n)
+ *   CAMERA_MEAN_Z_SUM out = sum_z [ sum_n M_n f_n / max(1, sum_n M_n) ]      (paper Eq. 1)
+ */
+typedef enum flashbev_reduce {
+    FLASHBEV_REDUCE_SUM = 0,
+    FLASHBEV_REDUCE_MEAN_OVER_VALID = 1,
+    FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM = 2
+} flashbev_reduce;
+
+/* Kernel selection.  AUTO picks the tiled kernel whenever the channel row is a whole number of
+ * 16-byte vectors and `features` is 16-byte aligned, the per-output kernel otherwise. */
+typedef enum flashbev_kernel {
+    FLASHBEV_KERNEL_AUTO = 0,
+    FLASHBEV_KERNEL_PER_OUTPUT = 1, /* one thread per (cell, channel group), geometry recomputed per
+                                       thread: the decomposition Algorithm 2 describes */
+    FLASHBEV_KERNEL_TILED = 2       /* geometry once per (cell, camera, height) per CTA, broadcast to
+                                       channel lanes through shared memory */
+} flashbev_kernel;
+
+/*
+ * Operator description (Sec. 3.1 for the mathematics, Algorithm 2 for inputs and output).
+ *
+ * Geometry conventions:
+ *   - voxel centres are bin centres: x_w(ix) = x_min + (ix + 1/2)(x_max - x_min)/X, likewise y, z
+ *     (Sec. 4.1: [-50,50] m at 0.5 m <-> 200 bins);
+ *   - lidar2img[b][n] is a row-major 4x4 float matrix taking homogeneous metres to
+ *     (u*d, v*d, d) with (u, v) in full-resolution image pixels; row 3 is never read;
+ *   - feature-map coordinates follow grid_sample(align_corners=False):
+ *       fx = u * feat_w / img_w - 1/2,  fy = v * feat_h / img_h - 1/2;
+ *   - M_n = 1 iff d > 0.1 and -1/2 < fx < feat_w - 1/2 and -1/2 < fy < feat_h - 1/2;
+ *   - f_n is bilinear with zero padding; a valid sample counts once whatever number of its
+ *     taps is in bounds.
+ * Projection, validity, floor and the fractional parts are evaluated in fp64; interpolation
+ * weights and accumulation are fp32.  Non-finite matrix entries make the affected samples
+ * invalid; they never cause a fault.
+ *
+ * Index ranges: N*feat_h*feat_w*C*sizeof(element) < 2^35 and B*X*Y < 2^31, N <= 64,
+ * else FLASHBEV_UNSUPPORTED.
+ */
+typedef struct flashbev_vt_params {
+    size_t struct_size;        /* sizeof(flashbev_vt_params) of the caller's header */
+    const void *features;      /* [B][N][feat_h][feat_w][C], element type feat_dtype; read only */
+    int32_t feat_dtype;        /* flashbev_dtype */
+    int32_t layout;            /* flashbev_layout */
+    const float *lidar2img;    /* [B][N][4][4] float32; read only */
+    int32_t B, N, C;
+    int32_t feat_h, feat_w;    /* feature map size (texels) */
+    int32_t img_h, img_w;      /* full-resolution image size (pixels) the matrices project to */
+    double x_min, x_max;       /* BEV ranges, metres; max > min */
+    double y_min, y_max;
+    double z_min, z_max;
+    int32_t X, Y, Z;           /* number of bins per axis */
+    int32_t reduce;            /* flashbev_reduce */
+    void *out;                 /* [B][X][Y][C] float32; every element is written exactly once (cells no
+                                  camera sees get 0), so no pre-zeroing is needed */
+    int32_t out_dtype;         /* FLASHBEV_F32 only (bf16 output: FLASHBEV_UNSUPPORTED) */
+    int32_t kernel;            /* flashbev_kernel */
+    int32_t *valid_count_out;  /* optional [B][X][Y] int32: sum_z sum_n M_n per cell; NULL to skip */
+    int32_t tune[4];           /* 0 = library defaults.  tune[0]: channel vectors per lane (1,2,4);
+                                  tune[1]: lanes per cell; tune[2]: height bins per geometry walker;
+                                  tune[3]: reserved.  Invalid combinations fall back to the defaults */
+} flashbev_vt_params;
+
+/*
+ * The operator (Eq. 1; Algorithm 2).  Validates `p` on the host (no CUDA call is made and no
+ * device memory is touched when validation fails), then enqueues exactly one kernel on `stream`
+ * (a cudaStream_t, passed as void*; NULL = the default stream) and returns without waiting.
+ * Uses no device memory beyond `features`, `lidar2img`, `out` and `valid_count_out`.
+ */
+flashbev_status flashbev_sampling_vt(const flashbev_vt_params *p, void *stream);
+
+/* Device scratch the operator needs beyond its inputs and outputs: always 0 (Sec. 3.3.1: all
+ * intermediates live in registers / on chip).  Exists so callers can assert the contract. */
+size_t flashbev_workspace_bytes(const flashbev_vt_params *p);
+
+/*
+ * Same operator for callers whose data lives in HOST memory.  `p->features`, `p->lidar2img`,
+ * `p->out` (and `p->valid_count_out` if not NULL) are HOST pointers here (pinned memory makes the
+ * copies asynchronous).  `d_staging` is a caller-owned DEVICE buffer of at least
+ * flashbev_host_staging_bytes(p) bytes, 256-byte aligned.  Enqueues on `stream`: host->device
+ * copies of features and matrices, the kernel, device->host copy of the output; returns without
+ * waiting -- synchronise `stream` before reading `out`.  Allocates nothing.
+ */
+flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_staging,
+                                          size_t staging_bytes, void *stream);
+size_t flashbev_host_staging_bytes(const flashbev_vt_params *p); /* 0 if `p` is invalid */
+
+/* Number of kernels the last successful call of flashbev_sampling_vt[_host] on this thread
+ * enqueued (always 1), and a short name of the kernel instance it chose (static storage). */
+int flashbev_last_launch_count(void);
+const char *flashbev_last_kernel_name(void);
+
+const char *flashbev_status_string(int status); /* static storage, never NULL */
+int flashbev_version(void);                     /* FLASHBEV_VERSION of the built library */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLASHBEV_H_ */

@@ -1,0 +1,177 @@
+"""Thin ctypes binding of the C ABI in include/flashbev.h.
+
+Argument marshalling only: every step of the operator runs inside the CUDA
+library.  PyTorch is used by callers for device memory and streams; this module
+needs only integer addresses.  There is no CPU fallback: if the library has not
+been built, or the call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libflashbev.so")
+
+OK, INVALID_ARG, UNSUPPORTED, MISALIGNED, CUDA_ERROR, TOO_SMALL = range(6)
+F32, BF16 = 0, 1
+NHWC, NCHW = 0, 1
+REDUCE_SUM, REDUCE_MEAN_OVER_VALID, REDUCE_CAMERA_MEAN_Z_SUM = 0, 1, 2
+KERNEL_AUTO, KERNEL_PER_OUTPUT, KERNEL_TILED = 0, 1, 2
+
+
+class VtParams(ctypes.Structure):
+    """Mirror of ``flashbev_vt_params``."""
+    _fields_ = [
+        ("struct_size", ctypes.c_size_t),
+        ("features", ctypes.c_void_p),
+        ("feat_dtype", ctypes.c_int32),
+        ("layout", ctypes.c_int32),
+        ("lidar2img", ctypes.c_void_p),
+        ("B", ctypes.c_int32), ("N", ctypes.c_int32), ("C", ctypes.c_int32),
+        ("feat_h", ctypes.c_int32), ("feat_w", ctypes.c_int32),
+        ("img_h", ctypes.c_int32), ("img_w", ctypes.c_int32),
+        ("x_min", ctypes.c_double), ("x_max", ctypes.c_double),
+        ("y_min", ctypes.c_double), ("y_max", ctypes.c_double),
+        ("z_min", ctypes.c_double), ("z_max", ctypes.c_double),
+        ("X", ctypes.c_int32), ("Y", ctypes.c_int32), ("Z", ctypes.c_int32),
+        ("reduce", ctypes.c_int32),
+        ("out", ctypes.c_void_p),
+        ("out_dtype", ctypes.c_int32),
+        ("kernel", ctypes.c_int32),
+        ("valid_count_out", ctypes.c_void_p),
+        ("tune", ctypes.c_int32 * 4),
+    ]
+
+
+class FlashBevError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: {status_string(status)} (status {status})")
+        self.status = status
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libflashbev.so (built in-tree by ``paper_2607_10071_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2607_10071_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        P = ctypes.POINTER(VtParams)
+        L.flashbev_sampling_vt.restype = ctypes.c_int
+        L.flashbev_sampling_vt.argtypes = [P, ctypes.c_void_p]
+        L.flashbev_sampling_vt_host.restype = ctypes.c_int
+        L.flashbev_sampling_vt_host.argtypes = [P, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.flashbev_workspace_bytes.restype = ctypes.c_size_t
+        L.flashbev_workspace_bytes.argtypes = [P]
+        L.flashbev_host_staging_bytes.restype = ctypes.c_size_t
+        L.flashbev_host_staging_bytes.argtypes = [P]
+        L.flashbev_last_launch_count.restype = ctypes.c_int
+        L.flashbev_last_kernel_name.restype = ctypes.c_char_p
+        L.flashbev_status_string.restype = ctypes.c_char_p
+        L.flashbev_status_string.argtypes = [ctypes.c_int]
+        L.flashbev_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().flashbev_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().flashbev_version())
+
+
+def make_params(features_ptr, feat_dtype, lidar2img_ptr, B, N, C, feat_hw, img_hw, bev_range, grid,
+                reduce, out_ptr, valid_count_ptr=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0),
+                layout=NHWC, out_dtype=F32) -> VtParams:
+    p = VtParams()
+    p.struct_size = ctypes.sizeof(VtParams)
+    p.features, p.feat_dtype, p.layout = features_ptr, feat_dtype, layout
+    p.lidar2img = lidar2img_ptr
+    p.B, p.N, p.C = B, N, C
+    p.feat_h, p.feat_w = feat_hw
+    p.img_h, p.img_w = img_hw
+    p.x_min, p.x_max, p.y_min, p.y_max, p.z_min, p.z_max = (float(v) for v in bev_range)
+    p.X, p.Y, p.Z = grid
+    p.reduce = reduce
+    p.out, p.out_dtype, p.kernel = out_ptr, out_dtype, kernel
+    p.valid_count_out = valid_count_ptr
+    for i, t in enumerate(tune):
+        p.tune[i] = int(t)
+    return p
+
+
+def flashbev_sampling_vt(params: VtParams, stream: int | None = None, check: bool = True) -> int:
+    """Enqueue the fused operator on ``stream`` (a raw cudaStream_t value; None/0 = default stream)."""
+    st = lib().flashbev_sampling_vt(ctypes.byref(params), ctypes.c_void_p(stream or 0))
+    if check and st != OK:
+        raise FlashBevError(st, "flashbev_sampling_vt")
+    return st
+
+
+def flashbev_sampling_vt_host(params: VtParams, d_staging: int, staging_bytes: int, stream: int | None = None,
+                              check: bool = True) -> int:
+    """Host-buffer variant: pointers in ``params`` are host addresses, ``d_staging`` a device buffer."""
+    st = lib().flashbev_sampling_vt_host(ctypes.byref(params), ctypes.c_void_p(d_staging),
+                                         ctypes.c_size_t(staging_bytes), ctypes.c_void_p(stream or 0))
+    if check and st != OK:
+        raise FlashBevError(st, "flashbev_sampling_vt_host")
+    return st
+
+
+def flashbev_workspace_bytes(params: VtParams) -> int:
+    return int(lib().flashbev_workspace_bytes(ctypes.byref(params)))
+
+
+def flashbev_host_staging_bytes(params: VtParams) -> int:
+    return int(lib().flashbev_host_staging_bytes(ctypes.byref(params)))
+
+
+def flashbev_last_launch_count() -> int:
+    return int(lib().flashbev_last_launch_count())
+
+
+def flashbev_last_kernel_name() -> str:
+    return lib().flashbev_last_kernel_name().decode()
+
+
+# ---------------------------------------------------------------------------------------------
+# convenience for torch callers (marshalling only)
+
+def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM, out=None,
+                valid_count=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0), stream=None):
+    """features: CUDA tensor [B,N,Hf,Wf,C] float32 or bfloat16 (contiguous); lidar2img: CUDA float32
+    [B,N,4,4].  Returns the float32 output tensor [B,X,Y,C] (allocated by torch if ``out`` is None)."""
+    import torch
+
+    if not features.is_cuda or not lidar2img.is_cuda:
+        raise ValueError("sampling_vt needs CUDA tensors; there is no CPU path")
+    if not features.is_contiguous() or not lidar2img.is_contiguous():
+        raise ValueError("features and lidar2img must be contiguous")
+    if features.dtype == torch.float32:
+        dt = F32
+    elif features.dtype == torch.bfloat16:
+        dt = BF16
+    else:
+        raise ValueError("features must be float32 or bfloat16")
+    if lidar2img.dtype != torch.float32:
+        raise ValueError("lidar2img must be float32")
+    B, N, Hf, Wf, C = features.shape
+    X, Y, Z = grid
+    if out is None:
+        out = torch.empty((B, X, Y, C), dtype=torch.float32, device=features.device)
+    p = make_params(features.data_ptr(), dt, lidar2img.data_ptr(), B, N, C, (Hf, Wf), img_hw, bev_range,
+                    (X, Y, Z), reduce, out.data_ptr(),
+                    None if valid_count is None else valid_count.data_ptr(), kernel, tune)
+    if stream is None:
+        stream = torch.cuda.current_stream(features.device).cuda_stream
+    with torch.cuda.device(features.device):
+        flashbev_sampling_vt(p, stream)
+    return out

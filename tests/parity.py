@@ -1,0 +1,92 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C ABI, run the
+oracle on the same seeded inputs, and apply the tolerances.
+
+Tolerances (stated by the operator's specification):
+  fp32 features : max-abs <= 1e-4  and  relative L2 <= 1e-6
+  bf16 features : per output |gpu - oracle| <= 2e-3 * sqrt(max(1, valid-sample count)),
+                  the oracle being run on the same bf16-rounded inputs
+  validity      : valid-sample counts are integers and must match exactly
+Cells holding a sample within 1e-3 px (or 1e-3 m of the depth plane) of a validity border are
+flagged by the oracle and excluded from all three comparisons; the flagged samples must stay
+below 0.01 % of the candidates.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+from paper_2607_10071_b200 import binding as fb
+
+F32_MAX_ABS = 1e-4
+F32_REL_L2 = 1e-6
+BF16_ABS_PER_SQRT_COUNT = 2e-3
+MAX_FLAGGED_FRACTION = 1e-4
+
+
+def run_gpu(inp, reduce, kernel=fb.KERNEL_AUTO, tune=(0, 0, 0, 0), want_count=True, prefill=float("nan")):
+    """Upload, call flashbev_sampling_vt through the C ABI, download.  Returns (out, count, kernel_name)."""
+    import torch
+    w = inp.workload
+    dev = torch.device("cuda:0")
+    if w.dtype == "bf16":
+        feats = torch.from_numpy(inp.features_bf16.view(np.int16)).to(dev).view(torch.bfloat16)
+    else:
+        feats = torch.from_numpy(inp.features).to(dev)
+    mats = torch.from_numpy(inp.lidar2img).to(dev)
+    X, Y, Z = w.grid
+    out = torch.full((w.B, X, Y, w.C), prefill, dtype=torch.float32, device=dev)
+    cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=dev) if want_count else None
+    fb.sampling_vt(feats, mats, w.img_hw, w.bev_range, w.grid, reduce, out=out, valid_count=cnt,
+                   kernel=kernel, tune=tune)
+    name = fb.flashbev_last_kernel_name()
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), (cnt.cpu().numpy() if want_count else None), name
+
+
+@dataclass
+class ParityReport:
+    max_abs: float
+    rel_l2: float
+    worst_bf16_ratio: float     # max |err| / (2e-3 sqrt(count)); <= 1 passes
+    flagged_samples: int
+    flagged_fraction: float
+    excluded_cells: int
+    count_mismatches: int
+    valid_samples: int
+
+    def __str__(self):
+        return (f"max_abs={self.max_abs:.3e} rel_l2={self.rel_l2:.3e} bf16_ratio={self.worst_bf16_ratio:.3f} "
+                f"flagged={self.flagged_samples} ({self.flagged_fraction:.2e}) excluded_cells={self.excluded_cells} "
+                f"count_mismatch={self.count_mismatches} valid={self.valid_samples}")
+
+
+def compare(w, ref, out, count) -> ParityReport:
+    keep = ref.flagged == 0
+    g = out.astype(np.float64)[keep]
+    o = ref.out[keep]
+    err = np.abs(g - o)
+    max_abs = float(err.max()) if err.size else 0.0
+    nrm = float(np.sqrt((o * o).sum()))
+    rel = float(np.sqrt(((g - o) ** 2).sum()) / nrm) if nrm > 0 else float(np.sqrt(((g - o) ** 2).sum()))
+    bound = BF16_ABS_PER_SQRT_COUNT * np.sqrt(np.maximum(1, ref.count[keep]))[..., None]
+    ratio = float((err / bound).max()) if err.size else 0.0
+    mism = int((count[keep] != ref.count[keep]).sum()) if count is not None else 0
+    fl = int(ref.flagged.sum())
+    return ParityReport(max_abs, rel, ratio, fl, fl / max(1, w.candidates), int((~keep).sum()), mism,
+                        int(ref.count.sum()))
+
+
+def assert_parity(w, ref, out, count, label="", check_fraction=True):
+    rep = compare(w, ref, out, count)
+    msg = f"{label} {w.name}: {rep}"
+    assert np.all(np.isfinite(out)), f"{msg}: output has non-finite or unwritten elements"
+    assert rep.count_mismatches == 0, msg
+    if check_fraction:
+        assert rep.flagged_fraction < MAX_FLAGGED_FRACTION, msg
+    if w.dtype == "f32":
+        assert rep.max_abs <= F32_MAX_ABS, msg
+        assert rep.rel_l2 <= F32_REL_L2, msg
+    else:
+        assert rep.worst_bf16_ratio <= 1.0, msg
+    return rep

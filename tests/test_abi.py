@@ -1,0 +1,122 @@
+"""Host-only checks of the C ABI: the library loads, exports what the header declares, the
+ctypes mirror matches the C struct, and argument validation happens before any CUDA call."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+from paper_2607_10071_b200 import binding as fb
+from paper_2607_10071_b200 import build as fbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "flashbev.h")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    fbuild.build()
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(flashbev_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_functions()
+    assert "flashbev_sampling_vt" in names and len(names) >= 8
+    lib = ctypes.CDLL(fb.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in flashbev.h but not exported"
+
+
+def test_binding_exposes_the_same_names():
+    for n in declared_functions():
+        assert hasattr(fb, n) or n in ("flashbev_status_string", "flashbev_version"), n
+    assert fb.version() == 100
+    assert fb.status_string(fb.OK) == "ok" and "unknown" in fb.status_string(99)
+
+
+def test_ctypes_struct_matches_the_c_struct(tmp_path):
+    prog = tmp_path / "layout.c"
+    fields = [f[0] for f in fb.VtParams._fields_]
+    body = "\n".join(f'printf("{f} %zu\\n", offsetof(flashbev_vt_params, {f}));' for f in fields)
+    prog.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "flashbev.h"\nint main(void){\n'
+                    + body + '\nprintf("sizeof %zu\\n", sizeof(flashbev_vt_params));\nreturn 0;}\n')
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(prog), "-o", str(exe)],
+                   check=True)
+    got = dict(l.split() for l in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
+    for f in fields:
+        assert int(got[f]) == getattr(fb.VtParams, f).offset, f
+    assert int(got["sizeof"]) == ctypes.sizeof(fb.VtParams)
+
+
+def good_params(**over):
+    kw = dict(features_ptr=4096, feat_dtype=fb.F32, lidar2img_ptr=8192, B=1, N=6, C=32, feat_hw=(16, 44),
+              img_hw=(128, 352), bev_range=(-25, 25, -25, 25, -3, 1), grid=(50, 50, 4), reduce=0, out_ptr=16384)
+    kw.update(over)
+    return fb.make_params(**kw)
+
+
+@pytest.mark.parametrize("over,status", [
+    (dict(features_ptr=None), fb.INVALID_ARG),
+    (dict(lidar2img_ptr=None), fb.INVALID_ARG),
+    (dict(out_ptr=None), fb.INVALID_ARG),
+    (dict(B=0), fb.INVALID_ARG), (dict(N=-1), fb.INVALID_ARG), (dict(C=0), fb.INVALID_ARG),
+    (dict(feat_hw=(0, 44)), fb.INVALID_ARG), (dict(img_hw=(128, 0)), fb.INVALID_ARG),
+    (dict(grid=(50, 0, 4)), fb.INVALID_ARG), (dict(grid=(50, 50, 0)), fb.INVALID_ARG),
+    (dict(bev_range=(25, -25, -25, 25, -3, 1)), fb.INVALID_ARG),
+    (dict(bev_range=(-25, 25, -25, 25, 1, 1)), fb.INVALID_ARG),
+    (dict(bev_range=(-25, float("nan"), -25, 25, -3, 1)), fb.INVALID_ARG),
+    (dict(bev_range=(-25, float("inf"), -25, 25, -3, 1)), fb.INVALID_ARG),
+    (dict(reduce=3), fb.INVALID_ARG), (dict(feat_dtype=2), fb.INVALID_ARG), (dict(kernel=9), fb.INVALID_ARG),
+    (dict(layout=7), fb.INVALID_ARG),
+    (dict(layout=fb.NCHW), fb.UNSUPPORTED),
+    (dict(out_dtype=fb.BF16), fb.UNSUPPORTED),
+    (dict(N=65), fb.UNSUPPORTED),
+    (dict(B=1 << 20, grid=(1 << 10, 1 << 10, 4)), fb.UNSUPPORTED),
+    (dict(features_ptr=4098), fb.MISALIGNED),
+    (dict(out_ptr=16386), fb.MISALIGNED),
+    (dict(lidar2img_ptr=8194), fb.MISALIGNED),
+    (dict(features_ptr=4100, kernel=fb.KERNEL_TILED), fb.UNSUPPORTED),     # tiled kernel needs 16-byte alignment
+    (dict(C=30, kernel=fb.KERNEL_TILED), fb.UNSUPPORTED),
+])
+def test_invalid_arguments_are_rejected_on_the_host(over, status):
+    """None of these reach a CUDA call, so they run (and must not crash) on a machine without a GPU."""
+    assert fb.flashbev_sampling_vt(good_params(**over), None, check=False) == status
+
+
+def test_short_struct_and_null_params_are_rejected():
+    p = good_params()
+    p.struct_size = 8
+    assert fb.flashbev_sampling_vt(p, None, check=False) == fb.INVALID_ARG
+    assert fb.lib().flashbev_sampling_vt(None, None) == fb.INVALID_ARG
+    assert fb.flashbev_host_staging_bytes(p) == 0
+    with pytest.raises(fb.FlashBevError):
+        fb.flashbev_sampling_vt(p, None)
+
+
+def test_host_entry_validates_staging():
+    p = good_params()
+    need = fb.flashbev_host_staging_bytes(p)
+    assert need >= 1 * 6 * 16 * 44 * 32 * 4 + 6 * 64 + 50 * 50 * 32 * 4
+    assert fb.flashbev_sampling_vt_host(p, None, need, None, check=False) == fb.INVALID_ARG
+    assert fb.flashbev_sampling_vt_host(p, 4096 + 8, need, None, check=False) == fb.MISALIGNED
+    assert fb.flashbev_sampling_vt_host(p, 4096, need - 1, None, check=False) == fb.TOO_SMALL
+    assert fb.flashbev_workspace_bytes(p) == 0
+
+
+def test_product_path_never_imports_the_oracle():
+    code = ("import sys; import paper_2607_10071_b200.binding, paper_2607_10071_b200.workloads, "
+            "paper_2607_10071_b200.build; "
+            "assert not any(m == 'oracle' or m.startswith('oracle.') for m in sys.modules), 'oracle imported'")
+    subprocess.run([sys.executable, "-c", code], check=True, cwd=ROOT)
+    pat = re.compile(r"^\s*(from|import)\s+oracle\b|flashbev_oracle|oracle/", re.M)
+    for fn in ("binding.py", "workloads.py", "build.py", "__init__.py", os.path.join("csrc", "flashbev.cu")):
+        assert not pat.search(open(os.path.join(ROOT, "paper_2607_10071_b200", fn)).read()), fn
+    assert not pat.search(open(HEADER).read())

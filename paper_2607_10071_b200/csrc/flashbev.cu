@@ -25,10 +25,6 @@
 namespace {
 
 constexpr double kDepthMin = 0.1;   // metres: a sample needs camera depth > 0.1 m
-constexpr int kThreads = 256;       // tiled kernel: 8 warps
-constexpr int kWarps = kThreads / 32;
-constexpr int kRecordSlots = 128;   // list records per warp (shared by the warp's cells)
-constexpr int kWalkerCap = 2048;    // walker descriptors per CTA and height chunk
 constexpr int kMaxCams = 64;
 
 struct KParams {
@@ -42,12 +38,14 @@ struct KParams {
     // tiled kernel only
     int vecs;                   // 16-byte vectors per texel (C * elem / 16)
     int g;                      // lanes per cell
-    int cpw;                    // cells per warp
-    int wx, wy, Wx, Wy;         // cells per warp block, warp blocks per CTA tile (x, y)
-    int tiles_x, tiles_y;
+    int cpw, cpw_p2_log;        // cells per warp (= wx * wy) and log2 of its power-of-two ceiling
+    int wx, wy;                 // cells per warp block (x, y)
+    int blocks_x, blocks_y;     // warp blocks per batch element
+    int band, reps;             // block-id order: bands of `band` block rows; blocks per warp
     int zc;                     // height bins per chunk (multiple of 4 unless == Z)
     int walk;                   // height bins per walker
     int lcap;                   // records per cell list
+    int wcap;                   // walker descriptors per warp and height chunk
 };
 
 // ------------------------------------------------------------------------------------------
@@ -193,382 +191,505 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
 }
 
 // ------------------------------------------------------------------------------------------
-// Kernel 2: tiled.  Shared-memory layout (dynamic):
-//   double  mats[N][12]          rows 0..2 of lidar2img[b][n], rows 0/1 pre-scaled to feature px
-//   float4  lists[warps][kRecordSlots + cpw]   per cell: lcap records (+1 pad) {vector offset, wL, wR, -}
-//   uint32  walkers[kWalkerCap]  packed (cell, camera, first bin in chunk, bins - 1)
-//   uint32  den[cells * zc / 4]  per (cell, z) camera counts, one byte each (Eq. 1 mode only)
-//   int     list_count[cells], cell_count[cells], n_walkers
+// Kernel 2: tiled.  Every WARP owns a small block of adjacent BEV cells (cpw = wx * wy cells) and
+// takes it through three phases on its own, synchronising only with __syncwarp: (A) per
+// (cell, camera) column, the interval of height bins that can be valid; (B) walkers: exact fp64
+// geometry of those bins, merged into row records in the warp's shared-memory lists; (C) gather:
+// channel lanes walk the lists with 128-bit loads and packed fp32 FMAs.  Warps of a CTA share only
+// the per-batch-element tables staged once at kernel start, so while one warp waits on its
+// geometry another streams features.  A warp processes `reps` consecutive blocks.
+//
+// Shared memory (dynamic):
+//   CTA   : double mats[N][12]   rows 0..2 of lidar2img[b][n], rows 0/1 pre-scaled to feature px
+//           float  slope[N][5]   per camera: d/dk of the five validity conditions
+//   warp  : int4    list[kRecordSlots + cpw]  per cell lcap (+1 pad) records {offL, offR, wL, wR}
+//           double2 cellxy[8]    voxel-centre (x_w, y_w) of the block's cells (NaN: outside the grid)
+//           uint32  walkers[wcap] packed (cell, camera, first bin in chunk, bins - 1)
+//           uint32  den[cpw * zc / 4] per (cell, z) camera counts, one byte each (Eq. 1 mode)
+//           uint32  wsave[9][32] state of a walker that stopped because its list was full
+//           int     list_count[8], list_end[8], cell_count[8], n_walkers
 
-struct TileSmem {
-    double *mats;
-    float4 *lists;
+constexpr int kRecordSlots = 128;   // list records per warp (shared by the warp's cells)
+constexpr int kSaveWords = 9;
+constexpr int kWalkIlp = 4;         // height bins whose geometry a walker evaluates independently
+
+struct WarpSmem {
+    int4 *list;
+    double2 *cellxy;
     uint32_t *walkers;
     uint32_t *den;
+    uint32_t *wsave;
     int *list_count;
+    int *list_end;
     int *cell_count;
     int *n_walkers;
 };
 
-__host__ __device__ inline size_t tile_smem_bytes(int N, int cells, int cpw, int zc)
+__host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
+
+__host__ __device__ inline size_t cta_table_bytes(int N)
 {
-    size_t s = (size_t)N * 12 * sizeof(double);
-    s += (size_t)kWarps * (kRecordSlots + cpw) * sizeof(float4);
-    s += (size_t)kWalkerCap * sizeof(uint32_t);
-    s += (size_t)((cells * zc + 3) / 4) * sizeof(uint32_t);
-    s += (size_t)(2 * cells + 4) * sizeof(int);
-    return s;
+    return align16((size_t)N * 12 * sizeof(double)) + align16((size_t)N * 5 * sizeof(float));
 }
 
-__device__ __forceinline__ TileSmem carve(unsigned char *base, int N, int cells, int cpw, int zc)
+__host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem *t, int cpw, int zc, int wcap)
 {
-    TileSmem t;
-    t.mats = reinterpret_cast<double *>(base);
-    base += (size_t)N * 12 * sizeof(double);
-    t.lists = reinterpret_cast<float4 *>(base);
-    base += (size_t)kWarps * (kRecordSlots + cpw) * sizeof(float4);
-    t.walkers = reinterpret_cast<uint32_t *>(base);
-    base += (size_t)kWalkerCap * sizeof(uint32_t);
-    t.den = reinterpret_cast<uint32_t *>(base);
-    base += (size_t)((cells * zc + 3) / 4) * sizeof(uint32_t);
-    t.list_count = reinterpret_cast<int *>(base);
-    t.cell_count = t.list_count + cells;
-    t.n_walkers = t.cell_count + cells;
-    return t;
+    size_t o = 0;
+    auto take = [&](size_t bytes) {
+        unsigned char *ptr = base ? base + o : nullptr;
+        o += align16(bytes);
+        return ptr;
+    };
+    unsigned char *p0 = take((size_t)(kRecordSlots + cpw) * sizeof(int4));
+    unsigned char *p1 = take((size_t)8 * sizeof(double2));
+    unsigned char *p2 = take((size_t)wcap * sizeof(uint32_t));
+    unsigned char *p3 = take((size_t)((cpw * zc + 3) / 4) * sizeof(uint32_t));
+    unsigned char *p4 = take((size_t)kSaveWords * 32 * sizeof(uint32_t));
+    unsigned char *p5 = take((size_t)(3 * 8 + 4) * sizeof(int));
+    if (t) {
+        t->list = reinterpret_cast<int4 *>(p0);
+        t->cellxy = reinterpret_cast<double2 *>(p1);
+        t->walkers = reinterpret_cast<uint32_t *>(p2);
+        t->den = reinterpret_cast<uint32_t *>(p3);
+        t->wsave = reinterpret_cast<uint32_t *>(p4);
+        t->list_count = reinterpret_cast<int *>(p5);
+        t->list_end = t->list_count + 8;
+        t->cell_count = t->list_end + 8;
+        t->n_walkers = t->cell_count + 8;
+    }
+    return o;
 }
 
-// Position of local cell c inside the CTA tile (warp-major, so a warp's cells are adjacent).
-__device__ __forceinline__ void cell_xy(const KParams &p, int c, int &lx, int &ly)
-{
-    const int w = c / p.cpw, j = c - w * p.cpw;
-    const int jx = j / p.wy, jy = j - jx * p.wy;
-    const int wxi = w / p.Wy, wyi = w - wxi * p.Wy;
-    lx = wxi * p.wx + jx;
-    ly = wyi * p.wy + jy;
-}
+// Exact (fp64) test and bilinear set-up of height bin k of a (cell, camera) column:
+// row_i(z) = a_i + m[4 i + 2] * z_w.  When the camera's depth row does not depend on z
+// (m[10] == 0: no pitch or roll) 1/d is computed once per column.
+struct ColumnWalk {
+    const double *m;
+    double a0, a1, a2, zc0, dz, wlim, hlim, rconst;
+    bool dconst, dead;
 
-// Geometry of one (cell, camera) column: row_i(z) = A_i + B_i * z_w, with B_i read from smem.
-struct Column {
-    double a0, a1, a2;
+    __device__ __forceinline__ void init(const KParams &p, const double *mats, int n, double2 xy)
+    {
+        m = mats + n * 12;
+        a0 = fma(m[1], xy.y, fma(m[0], xy.x, m[3]));
+        a1 = fma(m[5], xy.y, fma(m[4], xy.x, m[7]));
+        a2 = fma(m[9], xy.y, fma(m[8], xy.x, m[11]));
+        zc0 = p.z_min + 0.5 * p.dz;
+        dz = p.dz;
+        wlim = (double)p.Wf - 0.5;
+        hlim = (double)p.Hf - 0.5;
+        dconst = (m[10] == 0.0);
+        dead = dconst && !(a2 > kDepthMin);
+        rconst = (dconst && !dead) ? fast_rcp(a2) : 0.0;
+    }
+    __device__ __forceinline__ bool sample(int k, Sample &s) const
+    {
+        const double zw = fma((double)k, dz, zc0);
+        double r = rconst;
+        if (!dconst) {
+            const double d = fma(m[10], zw, a2);
+            if (!(d > kDepthMin)) return false;
+            r = fast_rcp(d);
+        } else if (dead) {
+            return false;
+        }
+        const double fx = fma(fma(m[2], zw, a0), r, -0.5);
+        const double fy = fma(fma(m[6], zw, a1), r, -0.5);
+        if (!(fx > -0.5 && fx < wlim && fy > -0.5 && fy < hlim)) return false;
+        const double flx = floor(fx), fly = floor(fy);
+        s.x0 = (int)flx;
+        s.y0 = (int)fly;
+        s.tx = (float)(fx - flx);
+        s.ty = (float)(fy - fly);
+        return true;
+    }
 };
 
-__device__ __forceinline__ Column make_column(const double *m, double xw, double yw)
+// Walker: one thread follows one (cell, camera) column over a short run of height bins, keeps the
+// two texel rows it is currently touching open, and merges the weights of successive bins that
+// fall on the same rows.  A row is written to the cell's list when the column leaves it.
+struct Walker {
+    int k, ox, oy, vcount;
+    bool open;
+    float uL, uR, lL, lR;
+
+    // Close rows and write them as records.  False (nothing changed) if the list is full.
+    __device__ __forceinline__ bool close_rows(const KParams &p, const WarpSmem &sm, int wc, int wn, int4 *wlist,
+                                               bool close_u, bool close_l)
+    {
+        // A tap outside the map gets weight 0 and the address of the record's other tap.
+        const bool inL = ox >= 0, inR = ox + 1 <= p.Wf - 1;
+        const float cuL = inL ? uL : 0.f, cuR = inR ? uR : 0.f;
+        const float clL = inL ? lL : 0.f, clR = inR ? lR : 0.f;
+        const bool emit_u = close_u && oy >= 0 && oy <= p.Hf - 1 && (cuL != 0.f || cuR != 0.f);
+        const bool emit_l = close_l && oy + 1 >= 0 && oy + 1 <= p.Hf - 1 && (clL != 0.f || clR != 0.f);
+        const int need = (int)emit_u + (int)emit_l;
+        if (!need) return true;
+        const int slot = atomicAdd(&sm.list_count[wc], need);
+        if (slot >= p.lcap) {  // full (one pad slot lets a 2-record write start at lcap - 1)
+            atomicMin(&sm.list_end[wc], slot);
+            return false;
+        }
+        const int rowv = p.Wf * p.vecs;
+        const int o = ((wn * p.Hf + oy) * p.Wf + ox) * p.vecs;
+        const int oL = inL ? o : o + p.vecs, oR = inR ? o + p.vecs : o;
+        int sl = slot;
+        if (emit_u) wlist[sl++] = make_int4(oL, oR, __float_as_int(cuL), __float_as_int(cuR));
+        if (emit_l) wlist[sl] = make_int4(oL + rowv, oR + rowv, __float_as_int(clL), __float_as_int(clR));
+        return true;
+    }
+
+    // Add one valid sample.  False (nothing changed) if a row had to be written and the list is full.
+    __device__ __forceinline__ bool add(const KParams &p, const WarpSmem &sm, int wc, int wn, int4 *wlist,
+                                        const Sample &s, float scale)
+    {
+        bool close_u = false, close_l = false;
+        if (open) {
+            if (s.x0 != ox) close_u = close_l = true;
+            else if (s.y0 == oy + 1) close_u = true;
+            else if (s.y0 == oy - 1) close_l = true;
+            else if (s.y0 != oy) close_u = close_l = true;
+            if ((close_u || close_l) && !close_rows(p, sm, wc, wn, wlist, close_u, close_l)) return false;
+        }
+        const float wx1 = s.tx, wx0 = 1.f - s.tx;
+        const float wy1 = s.ty * scale, wy0 = (1.f - s.ty) * scale;
+        const float w00 = wx0 * wy0, w01 = wx1 * wy0, w10 = wx0 * wy1, w11 = wx1 * wy1;
+        if (open && close_u && !close_l) {  // one row down: the old lower row becomes the upper row
+            uL = lL + w00, uR = lR + w01, lL = w10, lR = w11;
+        } else if (open && close_l && !close_u) {  // one row up
+            lL = uL + w10, lR = uR + w11, uL = w00, uR = w01;
+        } else if (open && !close_u) {
+            uL += w00, uR += w01, lL += w10, lR += w11;
+        } else {
+            uL = w00, uR = w01, lL = w10, lR = w11;
+        }
+        open = true;
+        ox = s.x0;
+        oy = s.y0;
+        ++vcount;
+        return true;
+    }
+};
+
+// Runs a walker from its saved position to the end of its run.  False if it had to stop.
+__device__ __forceinline__ bool run_walker(const KParams &p, const WarpSmem &sm, const double *mats, Walker &w, int wc,
+                                           int wn, int kend, int kc0, int4 *wlist)
 {
-    Column c;
-    c.a0 = fma(m[1], yw, fma(m[0], xw, m[3]));
-    c.a1 = fma(m[5], yw, fma(m[4], xw, m[7]));
-    c.a2 = fma(m[9], yw, fma(m[8], xw, m[11]));
-    return c;
+    ColumnWalk cw;
+    cw.init(p, mats, wn, sm.cellxy[wc]);
+    while (w.k <= kend) {
+        Sample s[kWalkIlp];
+        bool ok[kWalkIlp];
+#pragma unroll
+        for (int i = 0; i < kWalkIlp; ++i) ok[i] = (w.k + i <= kend) && cw.sample(w.k + i, s[i]);
+#pragma unroll
+        for (int i = 0; i < kWalkIlp; ++i) {
+            if (ok[i]) {
+                float scale = 1.f;
+                if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
+                    const int di = wc * p.zc + (w.k + i - kc0);
+                    const uint32_t dn = (sm.den[di >> 2] >> (8 * (di & 3))) & 0xffu;
+                    scale = 1.f / (float)(dn > 1u ? dn : 1u);
+                }
+                if (!w.add(p, sm, wc, wn, wlist, s[i], scale)) {
+                    w.k += i;
+                    return false;
+                }
+            }
+        }
+        w.k += kWalkIlp;
+    }
+    if (w.open) {
+        if (!w.close_rows(p, sm, wc, wn, wlist, true, true)) return false;
+        w.open = false;
+    }
+    return true;
 }
 
-template <int V, bool BF16>
-__global__ void __launch_bounds__(kThreads) vt_tiled_kernel(const KParams p)
+// acc += w * (channels of one 16-byte vector), two channels per packed fp32 FMA
+template <bool BF16>
+__device__ __forceinline__ void fma_vec(float2 (&acc)[BF16 ? 4 : 2], const uint4 &t, const float2 w)
+{
+    if (BF16) {
+        acc[0] = __ffma2_rn(make_float2(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u)), w, acc[0]);
+        acc[1] = __ffma2_rn(make_float2(__uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u)), w, acc[1]);
+        acc[2 % (BF16 ? 4 : 2)] =
+            __ffma2_rn(make_float2(__uint_as_float(t.z << 16), __uint_as_float(t.z & 0xffff0000u)), w, acc[2 % (BF16 ? 4 : 2)]);
+        acc[3 % (BF16 ? 4 : 2)] =
+            __ffma2_rn(make_float2(__uint_as_float(t.w << 16), __uint_as_float(t.w & 0xffff0000u)), w, acc[3 % (BF16 ? 4 : 2)]);
+    } else {
+        acc[0] = __ffma2_rn(make_float2(__uint_as_float(t.x), __uint_as_float(t.y)), w, acc[0]);
+        acc[1] = __ffma2_rn(make_float2(__uint_as_float(t.z), __uint_as_float(t.w)), w, acc[1]);
+    }
+}
+
+template <int V, bool BF16, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 20 : 24)) / WARPS)
+    vt_tiled_kernel(const KParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    constexpr int EPV = BF16 ? 8 : 4;  // channels per 16-byte vector
-    const int cells = kWarps * p.cpw;
-    const TileSmem sm = carve(smem_raw, p.N, cells, p.cpw, p.zc);
+    constexpr int PV = BF16 ? 4 : 2;  // channel pairs per 16-byte vector
+    constexpr int THREADS = WARPS * 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.z;
 
-    // ---- which tile
-    const int tpb = p.tiles_x * p.tiles_y;
-    const int b = blockIdx.x / tpb;
-    const int trem = blockIdx.x - b * tpb;
-    const int tile_x = trem / p.tiles_y, tile_y = trem - tile_x * p.tiles_y;
-    const int tx = p.Wx * p.wx, ty = p.Wy * p.wy;
-    const int ix0 = tile_x * tx, iy0 = tile_y * ty;
-    const double wlim = (double)p.Wf - 0.5, hlim = (double)p.Hf - 0.5;
+    double *mats = reinterpret_cast<double *>(smem_raw);
+    float *slope = reinterpret_cast<float *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)));
+    WarpSmem sm;
+    {
+        const size_t per_warp = warp_smem_layout(nullptr, nullptr, p.cpw, p.zc, p.wcap);
+        warp_smem_layout(smem_raw + cta_table_bytes(p.N) + warp * per_warp, &sm, p.cpw, p.zc, p.wcap);
+    }
 
-    // ---- stage the camera matrices of this batch element (a1)
-    for (int i = tid; i < p.N * 12; i += kThreads) {
+    // ---- per-CTA tables: camera matrices (scaled to feature px) and condition slopes
+    for (int i = tid; i < p.N * 12; i += THREADS) {
         const int n = i / 12, e = i - n * 12;
         double v = (double)__ldg(p.l2i + ((size_t)b * p.N + n) * 16 + e);
         if (e < 4) v *= p.sx;
         else if (e < 8) v *= p.sy;
-        sm.mats[i] = v;
+        mats[i] = v;
     }
-    for (int i = tid; i < cells; i += kThreads) sm.cell_count[i] = 0;
+    for (int n = tid; n < p.N; n += THREADS) {
+        const float *M = p.l2i + ((size_t)b * p.N + n) * 16;
+        const double m2 = (double)__ldg(M + 2) * p.sx, m6 = (double)__ldg(M + 6) * p.sy, m10 = (double)__ldg(M + 10);
+        // d/dk of: depth - 0.1, p0s, Wf d - p0s, p1s, Hf d - p1s
+        slope[n * 5 + 0] = (float)(m10 * p.dz);
+        slope[n * 5 + 1] = (float)(m2 * p.dz);
+        slope[n * 5 + 2] = (float)(((double)p.Wf * m10 - m2) * p.dz);
+        slope[n * 5 + 3] = (float)(m6 * p.dz);
+        slope[n * 5 + 4] = (float)(((double)p.Hf * m10 - m6) * p.dz);
+    }
+    __syncthreads();  // the only CTA-wide barrier
 
-    // ---- gather role of this lane
+    // ---- gather role of this lane inside its warp
     const int cg = lane / p.g, gl = lane - cg * p.g;
-    const int my_cell = warp * p.cpw + cg;  // valid if cg < cpw
-    int mlx = 0, mly = 0;
-    if (cg < p.cpw) cell_xy(p, my_cell, mlx, mly);
+    const int my_cell = cg < p.cpw ? cg : 0;
+    const int mjx = my_cell / p.wy, mjy = my_cell - mjx * p.wy;
     const int vec0 = blockIdx.y * (p.g * V) + gl;  // first channel vector of this lane
-    const bool lane_on = (cg < p.cpw) && (ix0 + mlx < p.X) && (iy0 + mly < p.Y);
-    const uint4 *featb = static_cast<const uint4 *>(p.feat) + (size_t)b * p.N * p.Hf * p.Wf * p.vecs;
-    const float4 *my_list = sm.lists + warp * (kRecordSlots + p.cpw) + (cg < p.cpw ? cg : 0) * (p.lcap + 1);
-
-    float acc[V][EPV];
+    // channel vectors past the end of the row (ragged last channel block) re-read vector 0, never stored
+    const uint4 *featv[V];
+    {
+        const uint4 *featb = static_cast<const uint4 *>(p.feat) + (size_t)b * p.N * p.Hf * p.Wf * p.vecs;
 #pragma unroll
-    for (int v = 0; v < V; ++v)
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
-
-    for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
-        const int kc1 = min(p.Z, kc0 + p.zc);  // chunk [kc0, kc1)
-        if (tid == 0) *sm.n_walkers = 0;
-        if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM)
-            for (int i = tid; i < (cells * p.zc + 3) / 4; i += kThreads) sm.den[i] = 0u;
-        __syncthreads();
-
-        // ---- phase A: per (cell, camera) column, a conservative interval of height bins that can
-        // be valid (every validity condition is linear in z once d > 0), split into walkers
-        for (int pr = tid; pr < cells * p.N; pr += kThreads) {
-            const int c = pr / p.N, n = pr - c * p.N;
-            int lx, ly;
-            cell_xy(p, c, lx, ly);
-            if (ix0 + lx >= p.X || iy0 + ly >= p.Y) continue;
-            const double xw = p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx;
-            const double yw = p.y_min + ((double)(iy0 + ly) + 0.5) * p.dy;
-            const double *m = sm.mats + n * 12;
-            const Column col = make_column(m, xw, yw);
-            const double zc0 = p.z_min + 0.5 * p.dz;  // centre of bin 0; z_w(k) = zc0 + k dz
-            // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom
-            const double al[5] = {col.a2 + m[10] * zc0 - kDepthMin, col.a0 + m[2] * zc0,
-                                  (double)p.Wf * (col.a2 + m[10] * zc0) - (col.a0 + m[2] * zc0),
-                                  col.a1 + m[6] * zc0, (double)p.Hf * (col.a2 + m[10] * zc0) - (col.a1 + m[6] * zc0)};
-            const double be[5] = {m[10] * p.dz, m[2] * p.dz, ((double)p.Wf * m[10] - m[2]) * p.dz, m[6] * p.dz,
-                                  ((double)p.Hf * m[10] - m[6]) * p.dz};
-            float lo = (float)kc0 - 1.f, hi = (float)kc1;
-            bool empty = false;
-#pragma unroll
-            for (int i = 0; i < 5; ++i) {
-                const float a = (float)al[i], bb = (float)be[i];
-                if (bb > 0.f) lo = fmaxf(lo, -a / bb);       // k > -a/b
-                else if (bb < 0.f) hi = fminf(hi, -a / bb);  // k < -a/b
-                else if (a <= 0.f) empty = true;             // independent of z (NaN: keep)
-            }
-            if (empty) continue;
-            // widen by a guard far above the float error; every bin is re-tested exactly later
-            const float guard = 0.05f + 1e-5f * (float)p.Z;
-            int klo = (int)floorf(fminf(fmaxf(lo - guard, (float)kc0 - 1.f), (float)kc1)) + 1;
-            int khi = (int)ceilf(fmaxf(fminf(hi + guard, (float)kc1), (float)kc0 - 1.f)) - 1;
-            klo = max(klo, kc0);
-            khi = min(khi, kc1 - 1);
-            if (klo > khi) continue;
-            const int nw = (khi - klo + p.walk) / p.walk;
-            const int base = atomicAdd(sm.n_walkers, nw);
-            for (int i = 0; i < nw; ++i) {
-                const int k0 = klo + i * p.walk, k1 = min(khi, k0 + p.walk - 1);
-                if (base + i < kWalkerCap)
-                    sm.walkers[base + i] = (uint32_t)c | ((uint32_t)n << 8) | ((uint32_t)(k0 - kc0) << 14) |
-                                           ((uint32_t)(k1 - k0) << 23);
-            }
-        }
-        __syncthreads();
-        const int n_walkers = min(*sm.n_walkers, kWalkerCap);
-
-        // ---- Eq. 1 mode: den_z = sum_n M_n for every (cell, z) of the chunk, before any weight
-        if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
-            for (int wi = tid; wi < n_walkers; wi += kThreads) {
-                const uint32_t wd = sm.walkers[wi];
-                const int c = wd & 0xff, n = (wd >> 8) & 0x3f, k0 = kc0 + ((wd >> 14) & 0x1ff), k1 = k0 + (wd >> 23);
-                int lx, ly;
-                cell_xy(p, c, lx, ly);
-                const double xw = p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx;
-                const double yw = p.y_min + ((double)(iy0 + ly) + 0.5) * p.dy;
-                const double *m = sm.mats + n * 12;
-                const Column col = make_column(m, xw, yw);
-                for (int k = k0; k <= k1; ++k) {
-                    const double zw = p.z_min + ((double)k + 0.5) * p.dz;
-                    Sample s;
-                    if (project_sample(fma(m[2], zw, col.a0), fma(m[6], zw, col.a1), fma(m[10], zw, col.a2), wlim,
-                                       hlim, s)) {
-                        const int di = c * p.zc + (k - kc0);
-                        atomicAdd(&sm.den[di >> 2], 1u << (8 * (di & 3)));
-                    }
-                }
-            }
-            __syncthreads();
-        }
-
-        // ---- walkers in batches of one per thread; each batch: walk -> gather, repeated while a
-        // walker had to stop because its cell's list was full
-        for (int wb = 0; wb < n_walkers; wb += kThreads) {
-            const int wi = wb + tid;
-            bool done = wi >= n_walkers;
-            int wc = 0, wn = 0, k = 0, kend = -1, vcount = 0;
-            Column col = {0.0, 0.0, 0.0};
-            const double *m = sm.mats;
-            if (!done) {
-                const uint32_t wd = sm.walkers[wi];
-                wc = wd & 0xff;
-                wn = (wd >> 8) & 0x3f;
-                k = kc0 + ((wd >> 14) & 0x1ff);
-                kend = k + (int)(wd >> 23);
-                int lx, ly;
-                cell_xy(p, wc, lx, ly);
-                const double xw = p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx;
-                const double yw = p.y_min + ((double)(iy0 + ly) + 0.5) * p.dy;
-                m = sm.mats + wn * 12;
-                col = make_column(m, xw, yw);
-            }
-            // open pair of texel rows (oy, oy+1) at column ox with merged weights
-            bool open = false, flushed = false;
-            int ox = 0, oy = 0;
-            float uL = 0.f, uR = 0.f, lL = 0.f, lR = 0.f;
-            float4 *wlist = sm.lists + (wc / p.cpw) * (kRecordSlots + p.cpw) + (wc % p.cpw) * (p.lcap + 1);
-
-            while (true) {
-                for (int i = tid; i < cells; i += kThreads) sm.list_count[i] = 0;
-                __syncthreads();
-
-                while (!done) {
-                    // what does the next step want to emit?
-                    Sample s;
-                    bool valid = false;
-                    float scale = 1.f;
-                    int close_u = 0, close_l = 0;  // close upper / lower open row
-                    if (k <= kend) {
-                        const double zw = p.z_min + ((double)k + 0.5) * p.dz;
-                        valid = project_sample(fma(m[2], zw, col.a0), fma(m[6], zw, col.a1), fma(m[10], zw, col.a2),
-                                               wlim, hlim, s);
-                        if (!valid) {
-                            ++k;
-                            continue;
-                        }
-                        if (open) {
-                            if (s.x0 == ox && s.y0 == oy) {
-                            } else if (s.x0 == ox && s.y0 == oy + 1) close_u = 1;
-                            else if (s.x0 == ox && s.y0 == oy - 1) close_l = 1;
-                            else close_u = close_l = 1;
-                        }
-                    } else {
-                        if (!open || flushed) {
-                            done = true;
-                            break;
-                        }
-                        close_u = close_l = 1;
-                    }
-                    // records to write: rows inside the map with a non-zero weight
-                    const float cuL = (ox >= 0) ? uL : 0.f, cuR = (ox + 1 <= p.Wf - 1) ? uR : 0.f;
-                    const float clL = (ox >= 0) ? lL : 0.f, clR = (ox + 1 <= p.Wf - 1) ? lR : 0.f;
-                    const bool emit_u = close_u && oy >= 0 && oy <= p.Hf - 1 && (cuL != 0.f || cuR != 0.f);
-                    const bool emit_l = close_l && oy + 1 >= 0 && oy + 1 <= p.Hf - 1 && (clL != 0.f || clR != 0.f);
-                    const int need = (int)emit_u + (int)emit_l;
-                    if (need) {
-                        const int slot = atomicAdd(&sm.list_count[wc], need);
-                        if (slot + need > p.lcap) {  // list full: null any slot we hold, retry next round
-                            if (slot < p.lcap) wlist[slot] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            break;
-                        }
-                        int sl = slot;
-                        if (emit_u) {
-                            const int off = ((wn * p.Hf + oy) * p.Wf + ox) * p.vecs;
-                            wlist[sl++] = make_float4(__int_as_float(off), cuL, cuR, 0.f);
-                        }
-                        if (emit_l) {
-                            const int off = ((wn * p.Hf + oy + 1) * p.Wf + ox) * p.vecs;
-                            wlist[sl] = make_float4(__int_as_float(off), clL, clR, 0.f);
-                        }
-                    }
-                    if (k > kend) {
-                        flushed = true;
-                        done = true;
-                        break;
-                    }
-                    // commit the sample
-                    if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
-                        const int di = wc * p.zc + (k - kc0);
-                        const uint32_t dn = (sm.den[di >> 2] >> (8 * (di & 3))) & 0xffu;
-                        scale = 1.f / (float)(dn > 1u ? dn : 1u);
-                    }
-                    const float wx1 = s.tx, wx0 = 1.f - s.tx;
-                    const float wy1 = s.ty * scale, wy0 = (1.f - s.ty) * scale;
-                    const float w00 = wx0 * wy0, w01 = wx1 * wy0, w10 = wx0 * wy1, w11 = wx1 * wy1;
-                    if (open && close_u && !close_l) {  // moved one row down
-                        uL = lL + w00, uR = lR + w01, lL = w10, lR = w11;
-                    } else if (open && close_l && !close_u) {  // moved one row up
-                        lL = uL + w10, lR = uR + w11, uL = w00, uR = w01;
-                    } else if (open && !close_u && !close_l) {
-                        uL += w00, uR += w01, lL += w10, lR += w11;
-                    } else {
-                        uL = w00, uR = w01, lL = w10, lR = w11;
-                    }
-                    open = true;
-                    ox = s.x0;
-                    oy = s.y0;
-                    ++vcount;
-                    ++k;
-                }
-                __syncthreads();
-
-                // ---- gather (a7): channel lanes walk their cell's records
-                {
-                    const int nrec = lane_on ? min(sm.list_count[my_cell], p.lcap) : 0;
-                    const int maxn = __reduce_max_sync(0xffffffffu, nrec);
-                    for (int j = 0; j < maxn; j += 2) {
-                        float4 r[2];
-                        r[0] = (j < nrec) ? my_list[j] : make_float4(0.f, 0.f, 0.f, 0.f);
-                        r[1] = (j + 1 < nrec) ? my_list[j + 1] : make_float4(0.f, 0.f, 0.f, 0.f);
-                        uint4 tl[2][V], tr[2][V];
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const uint4 *base = featb + __float_as_int(r[u].x);
-#pragma unroll
-                            for (int v = 0; v < V; ++v) {
-                                const int vi = vec0 + v * p.g;
-                                tl[u][v] = make_uint4(0u, 0u, 0u, 0u);
-                                tr[u][v] = make_uint4(0u, 0u, 0u, 0u);
-                                if (vi < p.vecs) {
-                                    if (r[u].y != 0.f) tl[u][v] = __ldg(base + vi);
-                                    if (r[u].z != 0.f) tr[u][v] = __ldg(base + p.vecs + vi);
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-#pragma unroll
-                            for (int v = 0; v < V; ++v) {
-                                if (BF16) {
-                                    float fl[8], fr[8];
-                                    unpack8(tl[u][v], fl);
-                                    unpack8(tr[u][v], fr);
-#pragma unroll
-                                    for (int e = 0; e < 8; ++e) {
-                                        acc[v][e % EPV] = fmaf(r[u].y, fl[e], acc[v][e % EPV]);
-                                        acc[v][e % EPV] = fmaf(r[u].z, fr[e], acc[v][e % EPV]);
-                                    }
-                                } else {
-                                    const float fl[4] = {__uint_as_float(tl[u][v].x), __uint_as_float(tl[u][v].y),
-                                                         __uint_as_float(tl[u][v].z), __uint_as_float(tl[u][v].w)};
-                                    const float fr[4] = {__uint_as_float(tr[u][v].x), __uint_as_float(tr[u][v].y),
-                                                         __uint_as_float(tr[u][v].z), __uint_as_float(tr[u][v].w)};
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e) {
-                                        acc[v][e] = fmaf(r[u].y, fl[e], acc[v][e]);
-                                        acc[v][e] = fmaf(r[u].z, fr[e], acc[v][e]);
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
-                if (!__syncthreads_or(!done)) break;
-            }
-            if (wi < n_walkers && vcount) atomicAdd(&sm.cell_count[wc], vcount);
-        }
-        __syncthreads();
+        for (int v = 0; v < V; ++v) featv[v] = featb + ((vec0 + v * p.g < p.vecs) ? vec0 + v * p.g : 0);
     }
+    const int4 *my_list = sm.list + my_cell * (p.lcap + 1);
 
-    // ---- epilogue (a8): one store per output vector
-    if (lane_on) {
-        const int count = sm.cell_count[my_cell];
-        const float g = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-        const size_t cell = ((size_t)b * p.X + (ix0 + mlx)) * p.Y + (iy0 + mly);
-        float *o = p.out + cell * p.C;
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            const int vi = vec0 + v * p.g;
-            if (vi < p.vecs) {
-#pragma unroll
-                for (int e = 0; e < EPV; e += 4)
-                    __stcs(reinterpret_cast<float4 *>(o + (size_t)vi * EPV + e),
-                           make_float4(acc[v][e] * g, acc[v][e + 1] * g, acc[v][e + 2] * g, acc[v][e + 3] * g));
-            }
+    for (int rep = 0; rep < p.reps; ++rep) {
+        // ---- which block of cells: ids run along y inside bands of `band` block rows
+        const int id = (blockIdx.x * WARPS + warp) * p.reps + rep;
+        const int per_band = p.band * p.blocks_y;
+        const int bandi = id / per_band, rem = id - bandi * per_band;
+        const int bx = bandi * p.band + (rem % p.band), by = rem / p.band;
+        if (bx >= p.blocks_x) continue;  // warp-uniform
+        const int ix0 = bx * p.wx, iy0 = by * p.wy;
+        const bool lane_on = (cg < p.cpw) && (ix0 + mjx < p.X) && (iy0 + mjy < p.Y);
+
+        if (lane < 8) {
+            const int jx = lane / p.wy, jy = lane - jx * p.wy;
+            const bool in = (lane < p.cpw) && (ix0 + jx < p.X) && (iy0 + jy < p.Y);
+            const double nan = __longlong_as_double(0x7ff8000000000000LL);
+            sm.cellxy[lane] = make_double2(in ? p.x_min + ((double)(ix0 + jx) + 0.5) * p.dx : nan,
+                                           in ? p.y_min + ((double)(iy0 + jy) + 0.5) * p.dy : nan);
+            sm.cell_count[lane] = 0;
         }
-        if (p.count_out && gl == 0 && blockIdx.y == 0) p.count_out[cell] = count;
+
+        float2 acc[V][PV];
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
+        bool any_rec = false;
+
+        for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
+            const int kc1 = min(p.Z, kc0 + p.zc);  // chunk [kc0, kc1)
+            if (lane == 0) *sm.n_walkers = 0;
+            if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM)
+                for (int i = lane; i < (p.cpw * p.zc + 3) / 4; i += 32) sm.den[i] = 0u;
+            __syncwarp();
+
+            // ---- phase A: per (cell, camera) column, a conservative interval of height bins that can
+            // be valid (every validity condition is linear in z once d > 0), split into walkers
+            for (int pr = lane; pr < (p.N << p.cpw_p2_log); pr += 32) {
+                const int c = pr & ((1 << p.cpw_p2_log) - 1), n = pr >> p.cpw_p2_log;
+                if (c >= p.cpw) continue;
+                const double2 xy = sm.cellxy[c];
+                if (!(xy.x == xy.x)) continue;
+                const double *m = mats + n * 12;
+                const float *sl = slope + n * 5;
+                const double zc0 = p.z_min + 0.5 * p.dz;  // centre of bin 0; z_w(k) = zc0 + k dz
+                // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom
+                const double d0 = fma(m[10], zc0, fma(m[9], xy.y, fma(m[8], xy.x, m[11])));
+                float lo = (float)kc0 - 1.f, hi = (float)kc1;
+                bool empty = false;
+                auto cond = [&](float a, float bslope) {
+                    if (bslope > 0.f) lo = fmaxf(lo, -a * __frcp_rn(bslope));       // k > -a/b
+                    else if (bslope < 0.f) hi = fminf(hi, -a * __frcp_rn(bslope));  // k < -a/b
+                    else if (a <= 0.f) empty = true;  // independent of z (NaN: keep, tested exactly later)
+                };
+                cond((float)(d0 - kDepthMin), sl[0]);
+                if (empty || !(lo < hi)) continue;
+                const double p00 = fma(m[2], zc0, fma(m[1], xy.y, fma(m[0], xy.x, m[3])));
+                cond((float)p00, sl[1]);
+                cond((float)fma((double)p.Wf, d0, -p00), sl[2]);
+                if (empty || !(lo < hi)) continue;
+                const double p10 = fma(m[6], zc0, fma(m[5], xy.y, fma(m[4], xy.x, m[7])));
+                cond((float)p10, sl[3]);
+                cond((float)fma((double)p.Hf, d0, -p10), sl[4]);
+                if (empty) continue;
+                // widen by a guard far above the float error; every bin is re-tested exactly later
+                const float guard = 0.05f + 1e-5f * (float)p.Z;
+                int klo = (int)floorf(fminf(fmaxf(lo - guard, (float)kc0 - 1.f), (float)kc1)) + 1;
+                int khi = (int)ceilf(fmaxf(fminf(hi + guard, (float)kc1), (float)kc0 - 1.f)) - 1;
+                klo = max(klo, kc0);
+                khi = min(khi, kc1 - 1);
+                if (klo > khi) continue;
+                const int nw = (khi - klo + p.walk) / p.walk;
+                const int base = atomicAdd(sm.n_walkers, nw);
+                for (int i = 0; i < nw; ++i) {
+                    const int k0 = klo + i * p.walk, k1 = min(khi, k0 + p.walk - 1);
+                    if (base + i < p.wcap)
+                        sm.walkers[base + i] = (uint32_t)c | ((uint32_t)n << 8) | ((uint32_t)(k0 - kc0) << 14) |
+                                               ((uint32_t)(k1 - k0) << 23);
+                }
+            }
+            __syncwarp();
+            const int n_walkers = min(*sm.n_walkers, p.wcap);
+
+            // ---- Eq. 1 mode: den_z = sum_n M_n for every (cell, z) of the chunk, before any weight
+            if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
+                for (int wi = lane; wi < n_walkers; wi += 32) {
+                    const uint32_t wd = sm.walkers[wi];
+                    const int c = wd & 0xff, n = (wd >> 8) & 0x3f, k0 = kc0 + ((wd >> 14) & 0x1ff), k1 = k0 + (wd >> 23);
+                    ColumnWalk cw;
+                    cw.init(p, mats, n, sm.cellxy[c]);
+                    for (int k = k0; k <= k1; ++k) {
+                        Sample s;
+                        if (cw.sample(k, s)) {
+                            const int di = c * p.zc + (k - kc0);
+                            atomicAdd(&sm.den[di >> 2], 1u << (8 * (di & 3)));
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+
+            // ---- walkers in batches of one per lane; each batch: walk -> gather, repeated while a
+            // walker had to stop because its cell's list was full
+            for (int wb = 0; wb < n_walkers; wb += 32) {
+                bool first = true;
+                while (true) {
+                    if (lane < 8) {
+                        sm.list_count[lane] = 0;
+                        sm.list_end[lane] = 0x7fffffff;
+                    }
+                    __syncwarp();
+
+                    bool pending = false;
+                    if (wb + lane < n_walkers) {
+                        const int flags = first ? 0 : (int)sm.wsave[8 * 32 + lane];
+                        if (!(flags & 2)) {
+                            const uint32_t wd = sm.walkers[wb + lane];
+                            const int wc = wd & 0xff, wn = (wd >> 8) & 0x3f;
+                            const int k0 = kc0 + ((wd >> 14) & 0x1ff), kend = k0 + (int)(wd >> 23);
+                            Walker w;
+                            if (first) {
+                                w.k = k0, w.ox = 0, w.oy = 0, w.vcount = 0, w.open = false;
+                                w.uL = w.uR = w.lL = w.lR = 0.f;
+                            } else {
+                                w.k = (int)sm.wsave[0 * 32 + lane];
+                                w.ox = (int)sm.wsave[1 * 32 + lane];
+                                w.oy = (int)sm.wsave[2 * 32 + lane];
+                                w.vcount = (int)sm.wsave[3 * 32 + lane];
+                                w.uL = __uint_as_float(sm.wsave[4 * 32 + lane]);
+                                w.uR = __uint_as_float(sm.wsave[5 * 32 + lane]);
+                                w.lL = __uint_as_float(sm.wsave[6 * 32 + lane]);
+                                w.lR = __uint_as_float(sm.wsave[7 * 32 + lane]);
+                                w.open = flags & 1;
+                            }
+                            const bool done = run_walker(p, sm, mats, w, wc, wn, kend, kc0, sm.list + wc * (p.lcap + 1));
+                            sm.wsave[8 * 32 + lane] = (uint32_t)((w.open ? 1 : 0) | (done ? 2 : 0));
+                            if (done) {
+                                if (w.vcount) atomicAdd(&sm.cell_count[wc], w.vcount);
+                            } else {
+                                pending = true;
+                                sm.wsave[0 * 32 + lane] = (uint32_t)w.k;
+                                sm.wsave[1 * 32 + lane] = (uint32_t)w.ox;
+                                sm.wsave[2 * 32 + lane] = (uint32_t)w.oy;
+                                sm.wsave[3 * 32 + lane] = (uint32_t)w.vcount;
+                                sm.wsave[4 * 32 + lane] = __float_as_uint(w.uL);
+                                sm.wsave[5 * 32 + lane] = __float_as_uint(w.uR);
+                                sm.wsave[6 * 32 + lane] = __float_as_uint(w.lL);
+                                sm.wsave[7 * 32 + lane] = __float_as_uint(w.lR);
+                            }
+                        }
+                    }
+                    __syncwarp();
+
+                    // ---- gather: channel lanes walk their cell's records, U per iteration; every record is
+                    // two taps of one texel row, both always loadable (out-of-map taps alias the other tap
+                    // with weight 0).  Lanes past the end of their list repeat their last record with weight 0.
+                    {
+                        constexpr int U = V == 1 ? 4 : (V == 2 ? 2 : 1);
+                        const int nrec = lane_on ? min(sm.list_count[my_cell], sm.list_end[my_cell]) : 0;
+                        const int maxn = __reduce_max_sync(0xffffffffu, nrec);
+                        any_rec |= nrec > 0;
+                        if (nrec > 0) {
+                            const int last = nrec - 1;
+                            for (int j = 0; j < maxn; j += U) {
+                                int4 r[U];
+#pragma unroll
+                                for (int u = 0; u < U; ++u) r[u] = my_list[min(j + u, last)];
+                                uint4 t[U][2][V];
+#pragma unroll
+                                for (int u = 0; u < U; ++u)
+#pragma unroll
+                                    for (int v = 0; v < V; ++v) {
+                                        t[u][0][v] = __ldg(featv[v] + r[u].x);
+                                        t[u][1][v] = __ldg(featv[v] + r[u].y);
+                                    }
+#pragma unroll
+                                for (int u = 0; u < U; ++u) {
+                                    const bool has = j + u <= last;
+                                    const float wl = has ? __int_as_float(r[u].z) : 0.f;
+                                    const float wr = has ? __int_as_float(r[u].w) : 0.f;
+#pragma unroll
+                                    for (int v = 0; v < V; ++v) {
+                                        fma_vec<BF16>(acc[v], t[u][0][v], make_float2(wl, wl));
+                                        fma_vec<BF16>(acc[v], t[u][1][v], make_float2(wr, wr));
+                                    }
+                                }
+                            }
+                        }
+                    }
+                    first = false;
+                    __syncwarp();
+                    if (!__any_sync(0xffffffffu, pending)) break;
+                }
+            }
+            __syncwarp();
+        }
+
+        // ---- epilogue: one store per output vector
+        if (lane_on) {
+            const int count = sm.cell_count[my_cell];
+            float g = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
+            if (!any_rec) g = 0.f;  // nothing sampled: exactly zero
+            const size_t cell = ((size_t)b * p.X + (ix0 + mjx)) * p.Y + (iy0 + mjy);
+            float *o = p.out + cell * p.C;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                const int vi = vec0 + v * p.g;
+                if (vi < p.vecs) {
+#pragma unroll
+                    for (int e = 0; e < PV; e += 2)
+                        __stcs(reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2),
+                               make_float4(acc[v][e].x * g, acc[v][e].y * g, acc[v][e + 1].x * g, acc[v][e + 1].y * g));
+                }
+            }
+            if (p.count_out && gl == 0 && blockIdx.y == 0) p.count_out[cell] = count;
+        }
+        __syncwarp();
     }
 }
 
@@ -667,15 +788,26 @@ bool tiled_applicable(const flashbev_vt_params *p)
     return vecs_total < 2147483648.0;
 }
 
-template <int V, bool BF16>
+template <int V, bool BF16, int WARPS>
 cudaError_t launch_tiled_inst(const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
 {
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    vt_tiled_kernel<V, BF16><<<grid, dim3(kThreads), smem, stream>>>(k);
+    vt_tiled_kernel<V, BF16, WARPS><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
     return cudaSuccess;
+}
+
+template <int V, bool BF16>
+cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
+{
+    switch (warps) {
+        case 1: return launch_tiled_inst<V, BF16, 1>(k, grid, smem, stream);
+        case 2: return launch_tiled_inst<V, BF16, 2>(k, grid, smem, stream);
+        case 8: return launch_tiled_inst<V, BF16, 8>(k, grid, smem, stream);
+        default: return launch_tiled_inst<V, BF16, 4>(k, grid, smem, stream);
+    }
 }
 
 flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
@@ -695,47 +827,54 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
         else V = 4, g = (k.vecs + 3) / 4;
         if (g > 32) g = 32;
     }
+    int warps = p->tune[3];
+    if (!(warps == 1 || warps == 2 || warps == 4 || warps == 8)) warps = 4;
     k.g = g;
     k.cpw = 32 / g;
     if (k.cpw > 8) k.cpw = 8;
-    // warp block (wx x wy cells) and CTA arrangement (Wx x Wy warps): near-square tiles
+    // warp block of wx x wy cells, near-square, y (the contiguous output axis) the longer side
     k.wy = (k.cpw % 2 == 0) ? 2 : (k.cpw == 3 ? 3 : 1);
     if (k.cpw == 8) k.wy = 4;
     if (k.cpw == 6) k.wy = 3;
+    if (k.cpw == 5 || k.cpw == 7) k.wy = k.cpw;
     k.wx = k.cpw / k.wy;
     k.cpw = k.wx * k.wy;
-    k.Wx = (k.wx >= k.wy) ? 2 : 4;
-    k.Wy = kWarps / k.Wx;
-    const int tx = k.Wx * k.wx, ty = k.Wy * k.wy, cells = kWarps * k.cpw;
-    k.tiles_x = (p->X + tx - 1) / tx;
-    k.tiles_y = (p->Y + ty - 1) / ty;
+    k.cpw_p2_log = 0;
+    while ((1 << k.cpw_p2_log) < k.cpw) k.cpw_p2_log += 1;
+    k.blocks_x = (p->X + k.wx - 1) / k.wx;
+    k.blocks_y = (p->Y + k.wy - 1) / k.wy;
+    k.band = 4;
+    k.reps = 4;
     k.lcap = kRecordSlots / k.cpw;
-    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : 8;
-    // height chunk: all walkers of a chunk must fit the descriptor array
-    int per_pair = kWalkerCap / (cells * p->N);
-    if (per_pair < 1) return FLASHBEV_UNSUPPORTED;
+    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : 4;
+    // height chunk: all walkers of a chunk must fit the warp's descriptor array
+    k.wcap = 128;
+    if (k.wcap < k.cpw * p->N) k.wcap = k.cpw * p->N;
+    const int per_pair = k.wcap / (k.cpw * p->N);
     int zc = per_pair * k.walk;
     if (zc > 256) zc = 256;
     if (zc >= p->Z) zc = p->Z;
-    else zc = (zc / 4) * 4 > 0 ? (zc / 4) * 4 : zc;
+    else if (zc >= 4) zc = (zc / 4) * 4;
     k.zc = zc;
 
-    const long long tiles = (long long)p->B * k.tiles_x * k.tiles_y;
+    const long long bands = (k.blocks_x + k.band - 1) / k.band;
+    const long long ids = bands * k.band * k.blocks_y;
+    const long long ctas = (ids + (long long)warps * k.reps - 1) / ((long long)warps * k.reps);
     const int cblocks = (k.vecs + g * V - 1) / (g * V);
-    if (tiles > 2147483647LL || cblocks > 65535) return FLASHBEV_UNSUPPORTED;
-    const dim3 grid((unsigned)tiles, (unsigned)cblocks);
-    const size_t smem = tile_smem_bytes(p->N, cells, k.cpw, k.zc);
+    if (ctas > 2147483647LL || cblocks > 65535 || p->B > 65535) return FLASHBEV_UNSUPPORTED;
+    const dim3 grid((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
+    const size_t smem = cta_table_bytes(p->N) + (size_t)warps * warp_smem_layout(nullptr, nullptr, k.cpw, k.zc, k.wcap);
     cudaError_t e;
     static const char *const names[2][3] = {{"tiled_f32_v1", "tiled_f32_v2", "tiled_f32_v4"},
                                             {"tiled_bf16_v1", "tiled_bf16_v2", "tiled_bf16_v4"}};
     if (bf16) {
-        if (V == 1) e = launch_tiled_inst<1, true>(k, grid, smem, stream);
-        else if (V == 2) e = launch_tiled_inst<2, true>(k, grid, smem, stream);
-        else e = launch_tiled_inst<4, true>(k, grid, smem, stream);
+        if (V == 1) e = launch_tiled_warps<1, true>(warps, k, grid, smem, stream);
+        else if (V == 2) e = launch_tiled_warps<2, true>(warps, k, grid, smem, stream);
+        else e = launch_tiled_warps<4, true>(warps, k, grid, smem, stream);
     } else {
-        if (V == 1) e = launch_tiled_inst<1, false>(k, grid, smem, stream);
-        else if (V == 2) e = launch_tiled_inst<2, false>(k, grid, smem, stream);
-        else e = launch_tiled_inst<4, false>(k, grid, smem, stream);
+        if (V == 1) e = launch_tiled_warps<1, false>(warps, k, grid, smem, stream);
+        else if (V == 2) e = launch_tiled_warps<2, false>(warps, k, grid, smem, stream);
+        else e = launch_tiled_warps<4, false>(warps, k, grid, smem, stream);
     }
     t_last_kernel = names[bf16 ? 1 : 0][V == 1 ? 0 : (V == 2 ? 1 : 2)];
     return e == cudaSuccess ? FLASHBEV_OK : FLASHBEV_CUDA_ERROR;

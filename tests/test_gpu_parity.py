@@ -102,6 +102,9 @@ def test_ragged_and_tiny_grids(oracle, grid):
 @pytest.mark.parametrize("Z", [1, 2, 63, 64, 65, 130, 300])
 def test_height_bin_counts_span_several_chunks(oracle, Z):
     inp = small(Z, B=1, C=32, grid=(9, 11, Z), z=(-4.0, 4.0))
+    # hundreds of samples per cell: keep |out| of order one so that the absolute tolerance, which
+    # was stated for outputs of that size, stays meaningful (fp32 accumulation error scales with |out|)
+    inp.features *= np.float32(1.0 / 16.0)
     for reduce in (SUM, EQ1):
         check_small(oracle, inp, reduce)
 
@@ -120,6 +123,7 @@ def test_every_camera_sees_every_cell_many_heights(oracle):
     inp = wl.make_inputs(w)
     inp.lidar2img[:] = inp.lidar2img[:, :1]                 # eight copies of the forward camera
     inp.lidar2img[0, :, 0, 3] += np.arange(8, dtype=np.float32) * 3.0   # shifted by a few pixels each
+    inp.features *= np.float32(1.0 / 16.0)      # ~770 samples per cell: keep |out| of order one (see above)
     for reduce in (SUM, MEAN, EQ1):
         ref, _, _ = check_small(oracle, inp, reduce)
         assert ref.count.max() > 300
@@ -136,7 +140,7 @@ def test_tuning_knobs_do_not_change_results(oracle, tune):
 
 def test_no_camera_sees_anything(oracle):
     inp = small(9, B=1, C=32, general=False, rng_xy=4.0)
-    inp.lidar2img[:, :, 2, :] *= -1.0                       # every depth negative
+    inp.lidar2img[:, :, 2, :] = np.array([0.0, 0.0, 0.0, -1.0], np.float32)   # depth -1 m everywhere
     ref, out, _ = check_small(oracle, inp, EQ1)
     assert ref.count.sum() == 0 and np.all(out == 0.0)
 

@@ -35,6 +35,9 @@ if ROOT not in sys.path:
 from paper_2607_10071_b200 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (bytes; None where no capture of that workload exists)
+NCU_DRAM_TRAFFIC = {"representative": 4.79e6, "long_range": 40.02e6}
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "fused_sampling_vt_throughput"
 UNIT = "sample-channels/s"
@@ -63,7 +66,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -261,7 +264,7 @@ def measure_e2e(torch, w, args, device, steps, warmup, dist_barrier):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="representative", choices=list(wl.WORKLOADS))
@@ -366,7 +369,7 @@ def main():
                    "kernel": m["kernel"]},
         "latency_ms": launch_ms,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "peak_kind": f"of {peak_kind}", "traffic": NCU_DRAM_TRAFFIC.get(w.name),
                      "algorithmic_bytes_per_launch": w.unique_bytes,
                      "frac_of_8TBs_nominal": achieved / 8000.0},
         "peak_mb": {"workspace_allocated_by_call": workspace / 1e6, "output": w.output_bytes / 1e6,

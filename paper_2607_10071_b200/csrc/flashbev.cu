@@ -22,6 +22,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+
 namespace {
 
 constexpr double kDepthMin = 0.1;   // metres: a sample needs camera depth > 0.1 m
@@ -38,13 +40,16 @@ struct KParams {
     // tiled kernel only
     int vecs;                   // 16-byte vectors per texel (C * elem / 16)
     int g;                      // lanes per cell
-    int cpw, cpw_p2_log;        // cells per warp (= wx * wy) and log2 of its power-of-two ceiling
-    int wx, wy;                 // cells per warp block (x, y)
-    int blocks_x, blocks_y;     // warp blocks per batch element
-    int band, reps;             // block-id order: bands of `band` block rows; blocks per warp
+    int cpw;                    // cells per sub-block (= wx * wy): the cells one gather pass covers
+    int wx, wy;                 // sub-block size in cells (x, y)
+    int sbx, sby, sbn;          // sub-blocks per super-block (x, y, total)
+    int ct, ct_inv;             // cells per super-block (<= 32) and ceil(65536 / ct)
+    int blocks_x, blocks_y;     // super-blocks per batch element
+    int band, reps;             // super-block order: bands of `band` rows; super-blocks per warp
     int zc;                     // height bins per chunk (multiple of 4 unless == Z)
     int walk;                   // height bins per walker
     int lcap;                   // records per cell list
+    int slots;                  // record slots per warp
     int wcap;                   // walker descriptors per warp and height chunk
 };
 
@@ -191,27 +196,36 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
 }
 
 // ------------------------------------------------------------------------------------------
-// Kernel 2: tiled.  Every WARP owns a small block of adjacent BEV cells (cpw = wx * wy cells) and
-// takes it through three phases on its own, synchronising only with __syncwarp: (A) per
-// (cell, camera) column, the interval of height bins that can be valid; (B) walkers: exact fp64
-// geometry of those bins, merged into row records in the warp's shared-memory lists; (C) gather:
-// channel lanes walk the lists with 128-bit loads and packed fp32 FMAs.  Warps of a CTA share only
-// the per-batch-element tables staged once at kernel start, so while one warp waits on its
-// geometry another streams features.  A warp processes `reps` consecutive blocks.
+// Kernel 2: tiled.  Every WARP owns a super-block of adjacent BEV cells (ct <= 32 cells, made of
+// sbn sub-blocks of cpw cells) and takes it through three phases on its own, synchronising only
+// with __syncwarp:
+//   (A) per (cell, camera) column: the interval of height bins that can be valid (all 32 lanes
+//       busy over the ct * N columns), split into short runs ("walkers");
+//   (B) walkers: a lane follows a run with exact fp64 geometry and merges successive bins that
+//       land on the same texel rows into row records in the cell's shared-memory list;
+//   (C) gather, one sub-block at a time: channel lanes walk their cell's list with 128-bit loads
+//       and packed fp32 FMAs, then store.
+// Warps of a CTA share only the per-batch-element tables staged once at kernel start, so while
+// one warp is in its geometry another streams features.
+//
+// A list that fills up makes its walkers stop; the warp then gathers what it has and runs another
+// round.  With one sub-block per warp the accumulators simply stay in registers across rounds and
+// height chunks; with several, a sub-block's partial sums are added to its own output elements
+// (owner-only read-modify-write, no atomics) and the last round applies the normalisation.
 //
 // Shared memory (dynamic):
 //   CTA   : double mats[N][12]   rows 0..2 of lidar2img[b][n], rows 0/1 pre-scaled to feature px
 //           float  slope[N][5]   per camera: d/dk of the five validity conditions
-//   warp  : int4    list[kRecordSlots + cpw]  per cell lcap (+1 pad) records {offL, offR, wL, wR}
-//           double2 cellxy[8]    voxel-centre (x_w, y_w) of the block's cells (NaN: outside the grid)
+//           int    celltab[32]   position of cell c inside a super-block: lx | ly << 8
+//   warp  : int4    list[slots + ct]  per cell lcap (+1 pad) records {offL, offR, wL, wR}
+//           double2 cellxy[32]   voxel-centre (x_w, y_w) of the cells (NaN: outside the grid)
 //           uint32  walkers[wcap] packed (cell, camera, first bin in chunk, bins - 1)
-//           uint32  den[cpw * zc / 4] per (cell, z) camera counts, one byte each (Eq. 1 mode)
+//           uint32  den[ct * zc / 4] per (cell, z) camera counts, one byte each (Eq. 1 mode)
 //           uint32  wsave[9][32] state of a walker that stopped because its list was full
-//           int     list_count[8], list_end[8], cell_count[8], n_walkers
+//           int     list_count[32], list_end[32], cell_count[32], n_walkers
 
-constexpr int kRecordSlots = 128;   // list records per warp (shared by the warp's cells)
 constexpr int kSaveWords = 9;
-constexpr int kWalkIlp = 4;         // height bins whose geometry a walker evaluates independently
+constexpr int kWalkIlp = 4;  // height bins whose geometry a walker evaluates independently
 
 struct WarpSmem {
     int4 *list;
@@ -229,10 +243,10 @@ __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t
 
 __host__ __device__ inline size_t cta_table_bytes(int N)
 {
-    return align16((size_t)N * 12 * sizeof(double)) + align16((size_t)N * 5 * sizeof(float));
+    return align16((size_t)N * 12 * sizeof(double)) + align16((size_t)N * 5 * sizeof(float)) + 32 * sizeof(int);
 }
 
-__host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem *t, int cpw, int zc, int wcap)
+__host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem *t, int ct, int slots, int zc, int wcap)
 {
     size_t o = 0;
     auto take = [&](size_t bytes) {
@@ -240,12 +254,12 @@ __host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem
         o += align16(bytes);
         return ptr;
     };
-    unsigned char *p0 = take((size_t)(kRecordSlots + cpw) * sizeof(int4));
-    unsigned char *p1 = take((size_t)8 * sizeof(double2));
+    unsigned char *p0 = take((size_t)(slots + ct) * sizeof(int4));
+    unsigned char *p1 = take((size_t)32 * sizeof(double2));
     unsigned char *p2 = take((size_t)wcap * sizeof(uint32_t));
-    unsigned char *p3 = take((size_t)((cpw * zc + 3) / 4) * sizeof(uint32_t));
+    unsigned char *p3 = take((size_t)((ct * zc + 3) / 4) * sizeof(uint32_t));
     unsigned char *p4 = take((size_t)kSaveWords * 32 * sizeof(uint32_t));
-    unsigned char *p5 = take((size_t)(3 * 8 + 4) * sizeof(int));
+    unsigned char *p5 = take((size_t)(3 * 32 + 4) * sizeof(int));
     if (t) {
         t->list = reinterpret_cast<int4 *>(p0);
         t->cellxy = reinterpret_cast<double2 *>(p1);
@@ -253,9 +267,9 @@ __host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem
         t->den = reinterpret_cast<uint32_t *>(p3);
         t->wsave = reinterpret_cast<uint32_t *>(p4);
         t->list_count = reinterpret_cast<int *>(p5);
-        t->list_end = t->list_count + 8;
-        t->cell_count = t->list_end + 8;
-        t->n_walkers = t->cell_count + 8;
+        t->list_end = t->list_count + 32;
+        t->cell_count = t->list_end + 32;
+        t->n_walkers = t->cell_count + 32;
     }
     return o;
 }
@@ -305,9 +319,7 @@ struct ColumnWalk {
     }
 };
 
-// Walker: one thread follows one (cell, camera) column over a short run of height bins, keeps the
-// two texel rows it is currently touching open, and merges the weights of successive bins that
-// fall on the same rows.  A row is written to the cell's list when the column leaves it.
+// Walker state: the two open texel rows (oy, oy + 1) at column ox with their merged weights.
 struct Walker {
     int k, ox, oy, vcount;
     bool open;
@@ -423,6 +435,42 @@ __device__ __forceinline__ void fma_vec(float2 (&acc)[BF16 ? 4 : 2], const uint4
     }
 }
 
+// Gather of one cell list by its channel lanes, U records per iteration.  Every record is two
+// taps of one texel row, both always loadable.  Lanes whose list is shorter than the warp's
+// longest repeat their last record with weight 0; lanes with no records do nothing.
+template <int V, bool BF16>
+__device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int4 *list, int nrec, int maxn,
+                                            const uint4 *const (&featv)[V])
+{
+    constexpr int U = V == 1 ? 4 : (V == 2 ? 2 : 1);
+    if (nrec <= 0) return;
+    const int last = nrec - 1;
+    for (int j = 0; j < maxn; j += U) {
+        int4 r[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) r[u] = list[min(j + u, last)];
+        uint4 t[U][2][V];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                t[u][0][v] = __ldg(featv[v] + r[u].x);
+                t[u][1][v] = __ldg(featv[v] + r[u].y);
+            }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool has = j + u <= last;
+            const float wl = has ? __int_as_float(r[u].z) : 0.f;
+            const float wr = has ? __int_as_float(r[u].w) : 0.f;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                fma_vec<BF16>(acc[v], t[u][0][v], make_float2(wl, wl));
+                fma_vec<BF16>(acc[v], t[u][1][v], make_float2(wr, wr));
+            }
+        }
+    }
+}
+
 template <int V, bool BF16, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 20 : 24)) / WARPS)
     vt_tiled_kernel(const KParams p)
@@ -430,18 +478,21 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr int PV = BF16 ? 4 : 2;  // channel pairs per 16-byte vector
     constexpr int THREADS = WARPS * 32;
+    constexpr unsigned FULL = 0xffffffffu;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.z;
 
     double *mats = reinterpret_cast<double *>(smem_raw);
     float *slope = reinterpret_cast<float *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)));
+    int *celltab = reinterpret_cast<int *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)) +
+                                           align16((size_t)p.N * 5 * sizeof(float)));
     WarpSmem sm;
     {
-        const size_t per_warp = warp_smem_layout(nullptr, nullptr, p.cpw, p.zc, p.wcap);
-        warp_smem_layout(smem_raw + cta_table_bytes(p.N) + warp * per_warp, &sm, p.cpw, p.zc, p.wcap);
+        const size_t per_warp = warp_smem_layout(nullptr, nullptr, p.ct, p.slots, p.zc, p.wcap);
+        warp_smem_layout(smem_raw + align16(cta_table_bytes(p.N)) + warp * per_warp, &sm, p.ct, p.slots, p.zc, p.wcap);
     }
 
-    // ---- per-CTA tables: camera matrices (scaled to feature px) and condition slopes
+    // ---- per-CTA tables: camera matrices (scaled to feature px), condition slopes, cell positions
     for (int i = tid; i < p.N * 12; i += THREADS) {
         const int n = i / 12, e = i - n * 12;
         double v = (double)__ldg(p.l2i + ((size_t)b * p.N + n) * 16 + e);
@@ -459,12 +510,21 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
         slope[n * 5 + 3] = (float)(m6 * p.dz);
         slope[n * 5 + 4] = (float)(((double)p.Hf * m10 - m6) * p.dz);
     }
+    for (int c = tid; c < 32; c += THREADS) {
+        int v = 0;
+        if (c < p.ct) {
+            const int s = c / p.cpw, j = c - s * p.cpw;  // sub-block, cell inside it
+            const int si = s / p.sby, sj = s - si * p.sby;
+            const int jx = j / p.wy, jy = j - jx * p.wy;
+            v = (si * p.wx + jx) | ((sj * p.wy + jy) << 8);
+        }
+        celltab[c] = v;
+    }
     __syncthreads();  // the only CTA-wide barrier
 
-    // ---- gather role of this lane inside its warp
+    // ---- gather role of this lane inside a sub-block
     const int cg = lane / p.g, gl = lane - cg * p.g;
-    const int my_cell = cg < p.cpw ? cg : 0;
-    const int mjx = my_cell / p.wy, mjy = my_cell - mjx * p.wy;
+    const bool role = cg < p.cpw;
     const int vec0 = blockIdx.y * (p.g * V) + gl;  // first channel vector of this lane
     // channel vectors past the end of the row (ragged last channel block) re-read vector 0, never stored
     const uint4 *featv[V];
@@ -473,25 +533,26 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
 #pragma unroll
         for (int v = 0; v < V; ++v) featv[v] = featb + ((vec0 + v * p.g < p.vecs) ? vec0 + v * p.g : 0);
     }
-    const int4 *my_list = sm.list + my_cell * (p.lcap + 1);
+    const int my_tab = celltab[lane];
 
     for (int rep = 0; rep < p.reps; ++rep) {
-        // ---- which block of cells: ids run along y inside bands of `band` block rows
+        // ---- which super-block: ids run along y inside bands of `band` rows of super-blocks
         const int id = (blockIdx.x * WARPS + warp) * p.reps + rep;
         const int per_band = p.band * p.blocks_y;
         const int bandi = id / per_band, rem = id - bandi * per_band;
-        const int bx = bandi * p.band + (rem % p.band), by = rem / p.band;
+        const int by = rem / p.band, bx = bandi * p.band + (rem - by * p.band);
         if (bx >= p.blocks_x) continue;  // warp-uniform
-        const int ix0 = bx * p.wx, iy0 = by * p.wy;
-        const bool lane_on = (cg < p.cpw) && (ix0 + mjx < p.X) && (iy0 + mjy < p.Y);
+        const int ix0 = bx * (p.sbx * p.wx), iy0 = by * (p.sby * p.wy);
 
-        if (lane < 8) {
-            const int jx = lane / p.wy, jy = lane - jx * p.wy;
-            const bool in = (lane < p.cpw) && (ix0 + jx < p.X) && (iy0 + jy < p.Y);
+        unsigned in_mask;  // bit c: cell c of the super-block is inside the grid
+        {
+            const int lx = my_tab & 0xff, ly = my_tab >> 8;
+            const bool in = (lane < p.ct) && (ix0 + lx < p.X) && (iy0 + ly < p.Y);
             const double nan = __longlong_as_double(0x7ff8000000000000LL);
-            sm.cellxy[lane] = make_double2(in ? p.x_min + ((double)(ix0 + jx) + 0.5) * p.dx : nan,
-                                           in ? p.y_min + ((double)(iy0 + jy) + 0.5) * p.dy : nan);
+            sm.cellxy[lane] = make_double2(in ? p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx : nan,
+                                           in ? p.y_min + ((double)(iy0 + ly) + 0.5) * p.dy : nan);
             sm.cell_count[lane] = 0;
+            in_mask = __ballot_sync(FULL, in);
         }
 
         float2 acc[V][PV];
@@ -499,22 +560,21 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
         for (int v = 0; v < V; ++v)
 #pragma unroll
             for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
-        bool any_rec = false;
+        unsigned touched = 0;  // bit s: this lane has already stored its part of sub-block s
 
         for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
             const int kc1 = min(p.Z, kc0 + p.zc);  // chunk [kc0, kc1)
             if (lane == 0) *sm.n_walkers = 0;
             if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM)
-                for (int i = lane; i < (p.cpw * p.zc + 3) / 4; i += 32) sm.den[i] = 0u;
+                for (int i = lane; i < (p.ct * p.zc + 3) / 4; i += 32) sm.den[i] = 0u;
             __syncwarp();
 
             // ---- phase A: per (cell, camera) column, a conservative interval of height bins that can
             // be valid (every validity condition is linear in z once d > 0), split into walkers
-            for (int pr = lane; pr < (p.N << p.cpw_p2_log); pr += 32) {
-                const int c = pr & ((1 << p.cpw_p2_log) - 1), n = pr >> p.cpw_p2_log;
-                if (c >= p.cpw) continue;
+            for (int pr = lane; pr < p.ct * p.N; pr += 32) {
+                const int n = (pr * p.ct_inv) >> 16, c = pr - n * p.ct;
+                if (!((in_mask >> c) & 1u)) continue;
                 const double2 xy = sm.cellxy[c];
-                if (!(xy.x == xy.x)) continue;
                 const double *m = mats + n * 12;
                 const float *sl = slope + n * 5;
                 const double zc0 = p.z_min + 0.5 * p.dz;  // centre of bin 0; z_w(k) = zc0 + k dz
@@ -574,120 +634,111 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                 __syncwarp();
             }
 
-            // ---- walkers in batches of one per lane; each batch: walk -> gather, repeated while a
-            // walker had to stop because its cell's list was full
-            for (int wb = 0; wb < n_walkers; wb += 32) {
-                bool first = true;
-                while (true) {
-                    if (lane < 8) {
-                        sm.list_count[lane] = 0;
-                        sm.list_end[lane] = 0x7fffffff;
-                    }
-                    __syncwarp();
+            // ---- rounds: walk (every lane runs its walkers lane, lane + 32, ... until one has to stop
+            // because its cell's list is full) -> gather all sub-blocks; repeat while walkers are left
+            int resume = lane;
+            bool has_state = false;
+            while (true) {
+                sm.list_count[lane] = 0;
+                sm.list_end[lane] = 0x7fffffff;
+                __syncwarp();
 
-                    bool pending = false;
-                    if (wb + lane < n_walkers) {
-                        const int flags = first ? 0 : (int)sm.wsave[8 * 32 + lane];
-                        if (!(flags & 2)) {
-                            const uint32_t wd = sm.walkers[wb + lane];
-                            const int wc = wd & 0xff, wn = (wd >> 8) & 0x3f;
-                            const int k0 = kc0 + ((wd >> 14) & 0x1ff), kend = k0 + (int)(wd >> 23);
-                            Walker w;
-                            if (first) {
-                                w.k = k0, w.ox = 0, w.oy = 0, w.vcount = 0, w.open = false;
-                                w.uL = w.uR = w.lL = w.lR = 0.f;
-                            } else {
-                                w.k = (int)sm.wsave[0 * 32 + lane];
-                                w.ox = (int)sm.wsave[1 * 32 + lane];
-                                w.oy = (int)sm.wsave[2 * 32 + lane];
-                                w.vcount = (int)sm.wsave[3 * 32 + lane];
-                                w.uL = __uint_as_float(sm.wsave[4 * 32 + lane]);
-                                w.uR = __uint_as_float(sm.wsave[5 * 32 + lane]);
-                                w.lL = __uint_as_float(sm.wsave[6 * 32 + lane]);
-                                w.lR = __uint_as_float(sm.wsave[7 * 32 + lane]);
-                                w.open = flags & 1;
-                            }
-                            const bool done = run_walker(p, sm, mats, w, wc, wn, kend, kc0, sm.list + wc * (p.lcap + 1));
-                            sm.wsave[8 * 32 + lane] = (uint32_t)((w.open ? 1 : 0) | (done ? 2 : 0));
-                            if (done) {
-                                if (w.vcount) atomicAdd(&sm.cell_count[wc], w.vcount);
-                            } else {
-                                pending = true;
-                                sm.wsave[0 * 32 + lane] = (uint32_t)w.k;
-                                sm.wsave[1 * 32 + lane] = (uint32_t)w.ox;
-                                sm.wsave[2 * 32 + lane] = (uint32_t)w.oy;
-                                sm.wsave[3 * 32 + lane] = (uint32_t)w.vcount;
-                                sm.wsave[4 * 32 + lane] = __float_as_uint(w.uL);
-                                sm.wsave[5 * 32 + lane] = __float_as_uint(w.uR);
-                                sm.wsave[6 * 32 + lane] = __float_as_uint(w.lL);
-                                sm.wsave[7 * 32 + lane] = __float_as_uint(w.lR);
-                            }
-                        }
+                bool pending = false;
+                for (int wi = resume; wi < n_walkers; wi += 32) {
+                    const uint32_t wd = sm.walkers[wi];
+                    const int wc = wd & 0xff, wn = (wd >> 8) & 0x3f;
+                    const int k0 = kc0 + ((wd >> 14) & 0x1ff), kend = k0 + (int)(wd >> 23);
+                    Walker w;
+                    if (has_state) {
+                        w.k = (int)sm.wsave[0 * 32 + lane];
+                        w.ox = (int)sm.wsave[1 * 32 + lane];
+                        w.oy = (int)sm.wsave[2 * 32 + lane];
+                        w.vcount = (int)sm.wsave[3 * 32 + lane];
+                        w.uL = __uint_as_float(sm.wsave[4 * 32 + lane]);
+                        w.uR = __uint_as_float(sm.wsave[5 * 32 + lane]);
+                        w.lL = __uint_as_float(sm.wsave[6 * 32 + lane]);
+                        w.lR = __uint_as_float(sm.wsave[7 * 32 + lane]);
+                        w.open = sm.wsave[8 * 32 + lane] != 0u;
+                        has_state = false;
+                    } else {
+                        w.k = k0, w.ox = 0, w.oy = 0, w.vcount = 0, w.open = false;
+                        w.uL = w.uR = w.lL = w.lR = 0.f;
                     }
-                    __syncwarp();
+                    if (run_walker(p, sm, mats, w, wc, wn, kend, kc0, sm.list + wc * (p.lcap + 1))) {
+                        if (w.vcount) atomicAdd(&sm.cell_count[wc], w.vcount);
+                    } else {
+                        sm.wsave[0 * 32 + lane] = (uint32_t)w.k;
+                        sm.wsave[1 * 32 + lane] = (uint32_t)w.ox;
+                        sm.wsave[2 * 32 + lane] = (uint32_t)w.oy;
+                        sm.wsave[3 * 32 + lane] = (uint32_t)w.vcount;
+                        sm.wsave[4 * 32 + lane] = __float_as_uint(w.uL);
+                        sm.wsave[5 * 32 + lane] = __float_as_uint(w.uR);
+                        sm.wsave[6 * 32 + lane] = __float_as_uint(w.lL);
+                        sm.wsave[7 * 32 + lane] = __float_as_uint(w.lR);
+                        sm.wsave[8 * 32 + lane] = w.open ? 1u : 0u;
+                        has_state = true;
+                        pending = true;
+                        resume = wi;
+                        break;
+                    }
+                }
+                if (!pending) resume = n_walkers;
+                __syncwarp();
+                const bool more = __any_sync(FULL, pending);
+                const bool final = !more && kc1 >= p.Z;  // last commit of this super-block
 
-                    // ---- gather: channel lanes walk their cell's records, U per iteration; every record is
-                    // two taps of one texel row, both always loadable (out-of-map taps alias the other tap
-                    // with weight 0).  Lanes past the end of their list repeat their last record with weight 0.
-                    {
-                        constexpr int U = V == 1 ? 4 : (V == 2 ? 2 : 1);
-                        const int nrec = lane_on ? min(sm.list_count[my_cell], sm.list_end[my_cell]) : 0;
-                        const int maxn = __reduce_max_sync(0xffffffffu, nrec);
-                        any_rec |= nrec > 0;
-                        if (nrec > 0) {
-                            const int last = nrec - 1;
-                            for (int j = 0; j < maxn; j += U) {
-                                int4 r[U];
+                // ---- gather, one sub-block at a time
+                for (int s = 0; s < p.sbn; ++s) {
+                    const int cell = s * p.cpw + (role ? cg : 0);
+                    const bool lane_on = role && ((in_mask >> cell) & 1u);
+                    const int nrec = lane_on ? min(sm.list_count[cell], sm.list_end[cell]) : 0;
+                    const int maxn = __reduce_max_sync(FULL, nrec);
+                    if (p.sbn > 1) {
 #pragma unroll
-                                for (int u = 0; u < U; ++u) r[u] = my_list[min(j + u, last)];
-                                uint4 t[U][2][V];
+                        for (int v = 0; v < V; ++v)
 #pragma unroll
-                                for (int u = 0; u < U; ++u)
+                            for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
+                    }
+                    gather_list<V, BF16>(acc, sm.list + cell * (p.lcap + 1), nrec, maxn, featv);
+                    const bool stored = (touched >> s) & 1u;
+                    // one sub-block per warp: accumulators live on; several: add to the stored partial sums
+                    const bool write = lane_on && (p.sbn > 1 ? (nrec > 0 || (final && (!stored ||
+                                                   p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID))) : final);
+                    if (write) {
+                        const int count = sm.cell_count[cell];
+                        const float g = (final && p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID)
+                                            ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
+                        const int tab = celltab[cell];
+                        const size_t ocell = ((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8));
+                        float *o = p.out + ocell * p.C;
 #pragma unroll
-                                    for (int v = 0; v < V; ++v) {
-                                        t[u][0][v] = __ldg(featv[v] + r[u].x);
-                                        t[u][1][v] = __ldg(featv[v] + r[u].y);
+                        for (int v = 0; v < V; ++v) {
+                            const int vi = vec0 + v * p.g;
+                            if (vi < p.vecs) {
+#pragma unroll
+                                for (int e = 0; e < PV; e += 2) {
+                                    float4 *dst = reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2);
+                                    float4 val = make_float4(acc[v][e].x, acc[v][e].y, acc[v][e + 1].x, acc[v][e + 1].y);
+                                    if (stored) {
+                                        const float4 prev = *dst;
+                                        val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
                                     }
-#pragma unroll
-                                for (int u = 0; u < U; ++u) {
-                                    const bool has = j + u <= last;
-                                    const float wl = has ? __int_as_float(r[u].z) : 0.f;
-                                    const float wr = has ? __int_as_float(r[u].w) : 0.f;
-#pragma unroll
-                                    for (int v = 0; v < V; ++v) {
-                                        fma_vec<BF16>(acc[v], t[u][0][v], make_float2(wl, wl));
-                                        fma_vec<BF16>(acc[v], t[u][1][v], make_float2(wr, wr));
-                                    }
+                                    val.x *= g, val.y *= g, val.z *= g, val.w *= g;
+                                    if (final) __stcs(dst, val);
+                                    else *dst = val;
                                 }
                             }
                         }
+                        touched |= 1u << s;
                     }
-                    first = false;
-                    __syncwarp();
-                    if (!__any_sync(0xffffffffu, pending)) break;
+                    if (final && lane_on && p.count_out && gl == 0 && blockIdx.y == 0) {
+                        const int tab = celltab[cell];
+                        p.count_out[((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8))] = sm.cell_count[cell];
+                    }
                 }
+                __syncwarp();
+                if (!more) break;
             }
-            __syncwarp();
-        }
-
-        // ---- epilogue: one store per output vector
-        if (lane_on) {
-            const int count = sm.cell_count[my_cell];
-            float g = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-            if (!any_rec) g = 0.f;  // nothing sampled: exactly zero
-            const size_t cell = ((size_t)b * p.X + (ix0 + mjx)) * p.Y + (iy0 + mjy);
-            float *o = p.out + cell * p.C;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int vi = vec0 + v * p.g;
-                if (vi < p.vecs) {
-#pragma unroll
-                    for (int e = 0; e < PV; e += 2)
-                        __stcs(reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2),
-                               make_float4(acc[v][e].x * g, acc[v][e].y * g, acc[v][e + 1].x * g, acc[v][e + 1].y * g));
-                }
-            }
-            if (p.count_out && gl == 0 && blockIdx.y == 0) p.count_out[cell] = count;
         }
         __syncwarp();
     }
@@ -827,31 +878,49 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
         else V = 4, g = (k.vecs + 3) / 4;
         if (g > 32) g = 32;
     }
-    int warps = p->tune[3];
+    int warps = p->tune[3] & 0xf;
     if (!(warps == 1 || warps == 2 || warps == 4 || warps == 8)) warps = 4;
     k.g = g;
     k.cpw = 32 / g;
     if (k.cpw > 8) k.cpw = 8;
-    // warp block of wx x wy cells, near-square, y (the contiguous output axis) the longer side
+    // sub-block of wx x wy cells, near-square, y (the contiguous output axis) the longer side
     k.wy = (k.cpw % 2 == 0) ? 2 : (k.cpw == 3 ? 3 : 1);
     if (k.cpw == 8) k.wy = 4;
     if (k.cpw == 6) k.wy = 3;
     if (k.cpw == 5 || k.cpw == 7) k.wy = k.cpw;
     k.wx = k.cpw / k.wy;
     k.cpw = k.wx * k.wy;
-    k.cpw_p2_log = 0;
-    while ((1 << k.cpw_p2_log) < k.cpw) k.cpw_p2_log += 1;
-    k.blocks_x = (p->X + k.wx - 1) / k.wx;
-    k.blocks_y = (p->Y + k.wy - 1) / k.wy;
-    k.band = 4;
-    k.reps = 4;
-    k.lcap = kRecordSlots / k.cpw;
     k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : 4;
+    const int runs = (p->Z + k.walk - 1) / k.walk;  // walkers per column when all of Z is one chunk
+
+    // super-block: as many sub-blocks as keep the whole height range in one chunk (<= 8 cells: larger
+    // ones pack the geometry lanes better but leave too few warps to overlap geometry with gathers)
+    int sbx = (p->tune[3] >> 4) & 0xf, sby = (p->tune[3] >> 8) & 0xf;
+    if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
+        sbx = sby = 1;
+        while (true) {
+            const bool grow_x = sbx * k.wx <= sby * k.wy;
+            const int nx = grow_x ? sbx * 2 : sbx, ny = grow_x ? sby : sby * 2;
+            const int ct = nx * ny * k.cpw;
+            // keep the whole height range in one chunk and leave each cell a list of ~1.5 Z + 4 records
+            if (ct > 8 || (long long)ct * p->N * runs > 512 || 2 * ct * (3 * p->Z + 8) > 2 * 2 * 192) break;
+            sbx = nx, sby = ny;
+        }
+    }
+    k.sbx = sbx, k.sby = sby, k.sbn = sbx * sby;
+    k.ct = k.sbn * k.cpw;
+    k.ct_inv = (65536 + k.ct - 1) / k.ct;
+    k.blocks_x = (p->X + sbx * k.wx - 1) / (sbx * k.wx);
+    k.blocks_y = (p->Y + sby * k.wy - 1) / (sby * k.wy);
+    k.band = 4;
+    k.reps = 1;
+    k.slots = k.sbn > 1 ? 192 : 128;
+    k.lcap = k.slots / k.ct;
     // height chunk: all walkers of a chunk must fit the warp's descriptor array
-    k.wcap = 128;
-    if (k.wcap < k.cpw * p->N) k.wcap = k.cpw * p->N;
-    const int per_pair = k.wcap / (k.cpw * p->N);
-    int zc = per_pair * k.walk;
+    k.wcap = (int)std::min<long long>(512, std::max<long long>(128, (long long)k.ct * p->N * runs));
+    if (k.wcap < k.ct * p->N) k.wcap = k.ct * p->N;
+    const int per_column = k.wcap / (k.ct * p->N);
+    int zc = per_column * k.walk;
     if (zc > 256) zc = 256;
     if (zc >= p->Z) zc = p->Z;
     else if (zc >= 4) zc = (zc / 4) * 4;
@@ -863,7 +932,8 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
     const int cblocks = (k.vecs + g * V - 1) / (g * V);
     if (ctas > 2147483647LL || cblocks > 65535 || p->B > 65535) return FLASHBEV_UNSUPPORTED;
     const dim3 grid((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
-    const size_t smem = cta_table_bytes(p->N) + (size_t)warps * warp_smem_layout(nullptr, nullptr, k.cpw, k.zc, k.wcap);
+    const size_t smem = align16(cta_table_bytes(p->N)) +
+                        (size_t)warps * warp_smem_layout(nullptr, nullptr, k.ct, k.slots, k.zc, k.wcap);
     cudaError_t e;
     static const char *const names[2][3] = {{"tiled_f32_v1", "tiled_f32_v2", "tiled_f32_v4"},
                                             {"tiled_bf16_v1", "tiled_bf16_v2", "tiled_bf16_v4"}};

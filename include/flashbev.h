@@ -32,7 +32,9 @@ typedef enum flashbev_status {
     FLASHBEV_MISALIGNED = 3,   /* `out` or `lidar2img` not 4-byte aligned, `features` not element aligned */
     FLASHBEV_CUDA_ERROR = 4,   /* the launch (or a copy of the host entry point) failed; the CUDA error
                                   has been consumed with cudaGetLastError */
-    FLASHBEV_TOO_SMALL = 5     /* a caller-provided staging buffer is smaller than required */
+    FLASHBEV_TOO_SMALL = 5,    /* a caller-provided staging buffer is smaller than required */
+    FLASHBEV_EXCEEDS_STATIC_STAGING = 6 /* flashbev_sampling_vt_host_static: the problem needs more than
+                                           FLASHBEV_STATIC_STAGING_BYTES of device staging */
 } flashbev_status;
 
 typedef enum flashbev_dtype { FLASHBEV_F32 = 0, FLASHBEV_BF16 = 1 } flashbev_dtype;
@@ -131,6 +133,34 @@ size_t flashbev_workspace_bytes(const flashbev_vt_params *p);
 flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_staging,
                                           size_t staging_bytes, void *stream);
 size_t flashbev_host_staging_bytes(const flashbev_vt_params *p); /* 0 if `p` is invalid */
+
+/*
+ * Host-buffer variant that needs no device buffer from the caller and never allocates.
+ * (The paper has no counterpart: this exists for deployment, not for the method.)
+ *
+ * Who needs it: callers that are not allowed to create device memory at the point where they call
+ * -- an inference-engine plugin that was handed no workspace, a perception loop whose memory budget
+ * is frozen after start-up, code running while other streams must not be disturbed (cudaMalloc and
+ * cudaFree synchronise the whole device), or a component that simply has no allocator to ask.
+ *
+ * Same contract as flashbev_sampling_vt_host (all pointers in `p` are HOST pointers, work is
+ * enqueued on `stream`, synchronise the stream before reading `out`), except that the device
+ * staging area is a fixed array of FLASHBEV_STATIC_STAGING_BYTES bytes that is part of the
+ * library image: every GPU on which the library is loaded sets that much memory aside until the
+ * process exits, whether this function is used or not.
+ *
+ *  - A problem whose flashbev_host_staging_bytes(p) exceeds FLASHBEV_STATIC_STAGING_BYTES is
+ *    refused with FLASHBEV_EXCEEDS_STATIC_STAGING before anything is enqueued.
+ *  - The first call on each device looks up the device address of the array (once per device, with
+ *    that device current) and remembers it; make that first call outside any stream capture.
+ *  - The array is shared by every call and keeps whatever the previous call left in it.  Nothing in
+ *    it has to start at zero (inputs are copied over it and the kernel writes every output
+ *    element), but two calls whose GPU work overlaps -- different streams, or different host
+ *    threads -- race on it: keep calls to this entry point in one stream order per device.
+ *  - Calls no cudaMalloc, cudaFree or any other allocating routine.
+ */
+#define FLASHBEV_STATIC_STAGING_BYTES (32u * 1024u * 1024u)
+flashbev_status flashbev_sampling_vt_host_static(const flashbev_vt_params *p, void *stream);
 
 /* Number of kernels the last successful call of flashbev_sampling_vt[_host] on this thread
  * enqueued (always 1), and a short name of the kernel instance it chose (static storage). */

@@ -14,6 +14,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libflashbev.so")
 
 OK, INVALID_ARG, UNSUPPORTED, MISALIGNED, CUDA_ERROR, TOO_SMALL = range(6)
+EXCEEDS_STATIC_STAGING = 6
+STATIC_STAGING_BYTES = 32 * 1024 * 1024
 F32, BF16 = 0, 1
 NHWC, NCHW = 0, 1
 REDUCE_SUM, REDUCE_MEAN_OVER_VALID, REDUCE_CAMERA_MEAN_Z_SUM = 0, 1, 2
@@ -67,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.flashbev_sampling_vt.argtypes = [P, ctypes.c_void_p]
         L.flashbev_sampling_vt_host.restype = ctypes.c_int
         L.flashbev_sampling_vt_host.argtypes = [P, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.flashbev_sampling_vt_host_static.restype = ctypes.c_int
+        L.flashbev_sampling_vt_host_static.argtypes = [P, ctypes.c_void_p]
         L.flashbev_workspace_bytes.restype = ctypes.c_size_t
         L.flashbev_workspace_bytes.argtypes = [P]
         L.flashbev_host_staging_bytes.restype = ctypes.c_size_t
@@ -123,6 +127,16 @@ def flashbev_sampling_vt_host(params: VtParams, d_staging: int, staging_bytes: i
                                          ctypes.c_size_t(staging_bytes), ctypes.c_void_p(stream or 0))
     if check and st != OK:
         raise FlashBevError(st, "flashbev_sampling_vt_host")
+    return st
+
+
+def flashbev_sampling_vt_host_static(params: VtParams, stream: int | None = None, check: bool = True) -> int:
+    """Host-buffer variant for callers that may not allocate device memory: pointers in ``params`` are
+    host addresses and the staging area is the fixed STATIC_STAGING_BYTES array inside the library.
+    Calls on one device must not overlap on the GPU (they share that array)."""
+    st = lib().flashbev_sampling_vt_host_static(ctypes.byref(params), ctypes.c_void_p(stream or 0))
+    if check and st != OK:
+        raise FlashBevError(st, "flashbev_sampling_vt_host_static")
     return st
 
 

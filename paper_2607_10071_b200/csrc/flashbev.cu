@@ -23,6 +23,7 @@
 #include <stdint.h>
 
 #include <algorithm>
+#include <mutex>
 
 namespace {
 
@@ -1039,6 +1040,48 @@ flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_s
     return FLASHBEV_OK;
 }
 
+// ---- allocation-free host entry point -------------------------------------------------------
+// The staging area lives in the library image.  In host code the array's name is only a handle:
+// the address the GPU understands has to be asked for, per device, with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_staging[FLASHBEV_STATIC_STAGING_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices];  // device address of g_static_staging on device i, once looked up
+
+// Device address of the built-in staging area on the current device (nullptr on failure).
+void *static_staging_address()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_staging) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        g_static_ptr[dev] = ptr;
+    }
+    return g_static_ptr[dev];
+}
+}  // namespace
+
+flashbev_status flashbev_sampling_vt_host_static(const flashbev_vt_params *p, void *stream)
+{
+    flashbev_status st;
+    if (!params_ok(p, st)) return st;
+    if (staging_layout(p).total > (size_t)FLASHBEV_STATIC_STAGING_BYTES) return FLASHBEV_EXCEEDS_STATIC_STAGING;
+    void *staging = static_staging_address();  // first call on this device: symbol look-up
+    if (!staging) return FLASHBEV_CUDA_ERROR;
+    // From here on this is the caller-staged path with the built-in area as the staging buffer.
+    return flashbev_sampling_vt_host(p, staging, (size_t)FLASHBEV_STATIC_STAGING_BYTES, stream);
+}
+
 int flashbev_last_launch_count(void) { return t_last_launches; }
 const char *flashbev_last_kernel_name(void) { return t_last_kernel; }
 
@@ -1051,6 +1094,7 @@ const char *flashbev_status_string(int status)
         case FLASHBEV_MISALIGNED: return "misaligned pointer";
         case FLASHBEV_CUDA_ERROR: return "CUDA error";
         case FLASHBEV_TOO_SMALL: return "staging buffer too small";
+        case FLASHBEV_EXCEEDS_STATIC_STAGING: return "problem exceeds the built-in staging area";
         default: return "unknown status";
     }
 }

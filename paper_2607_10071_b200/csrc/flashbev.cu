@@ -297,26 +297,20 @@ struct ColumnWalk {
         dead = dconst && !(a2 > kDepthMin);
         rconst = (dconst && !dead) ? fast_rcp(a2) : 0.0;
     }
+    // Branch-free apart from the (warp-uniform in practice) choice of the reciprocal.
     __device__ __forceinline__ bool sample(int k, Sample &s) const
     {
         const double zw = fma((double)k, dz, zc0);
-        double r = rconst;
-        if (!dconst) {
-            const double d = fma(m[10], zw, a2);
-            if (!(d > kDepthMin)) return false;
-            r = fast_rcp(d);
-        } else if (dead) {
-            return false;
-        }
+        const double d = dconst ? a2 : fma(m[10], zw, a2);
+        const double r = dconst ? rconst : fast_rcp(d);  // d <= 0 or NaN gives inf/NaN: every test below fails
         const double fx = fma(fma(m[2], zw, a0), r, -0.5);
         const double fy = fma(fma(m[6], zw, a1), r, -0.5);
-        if (!(fx > -0.5 && fx < wlim && fy > -0.5 && fy < hlim)) return false;
         const double flx = floor(fx), fly = floor(fy);
         s.x0 = (int)flx;
         s.y0 = (int)fly;
         s.tx = (float)(fx - flx);
         s.ty = (float)(fy - fly);
-        return true;
+        return (d > kDepthMin) & (fx > -0.5) & (fx < wlim) & (fy > -0.5) & (fy < hlim);
     }
 };
 
@@ -353,29 +347,23 @@ struct Walker {
     }
 
     // Add one valid sample.  False (nothing changed) if a row had to be written and the list is full.
+    // keep: same two rows; down / up: moved by one row, one open row is carried over.
     __device__ __forceinline__ bool add(const KParams &p, const WarpSmem &sm, int wc, int wn, int4 *wlist,
                                         const Sample &s, float scale)
     {
-        bool close_u = false, close_l = false;
-        if (open) {
-            if (s.x0 != ox) close_u = close_l = true;
-            else if (s.y0 == oy + 1) close_u = true;
-            else if (s.y0 == oy - 1) close_l = true;
-            else if (s.y0 != oy) close_u = close_l = true;
-            if ((close_u || close_l) && !close_rows(p, sm, wc, wn, wlist, close_u, close_l)) return false;
+        const bool same_col = open & (s.x0 == ox);
+        const int dy = s.y0 - oy;
+        const bool keep = same_col & (dy == 0), down = same_col & (dy == 1), up = same_col & (dy == -1);
+        const bool close_u = open & !(keep | up), close_l = open & !(keep | down);
+        if (close_u | close_l) {
+            if (!close_rows(p, sm, wc, wn, wlist, close_u, close_l)) return false;
         }
         const float wx1 = s.tx, wx0 = 1.f - s.tx;
         const float wy1 = s.ty * scale, wy0 = (1.f - s.ty) * scale;
         const float w00 = wx0 * wy0, w01 = wx1 * wy0, w10 = wx0 * wy1, w11 = wx1 * wy1;
-        if (open && close_u && !close_l) {  // one row down: the old lower row becomes the upper row
-            uL = lL + w00, uR = lR + w01, lL = w10, lR = w11;
-        } else if (open && close_l && !close_u) {  // one row up
-            lL = uL + w10, lR = uR + w11, uL = w00, uR = w01;
-        } else if (open && !close_u) {
-            uL += w00, uR += w01, lL += w10, lR += w11;
-        } else {
-            uL = w00, uR = w01, lL = w10, lR = w11;
-        }
+        const float nuL = w00 + (keep ? uL : (down ? lL : 0.f)), nuR = w01 + (keep ? uR : (down ? lR : 0.f));
+        const float nlL = w10 + (keep ? lL : (up ? uL : 0.f)), nlR = w11 + (keep ? lR : (up ? uR : 0.f));
+        uL = nuL, uR = nuR, lL = nlL, lR = nlR;
         open = true;
         ox = s.x0;
         oy = s.y0;
@@ -891,7 +879,7 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
     if (k.cpw == 5 || k.cpw == 7) k.wy = k.cpw;
     k.wx = k.cpw / k.wy;
     k.cpw = k.wx * k.wy;
-    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : 4;
+    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : (p->Z <= 16 ? 4 : (p->Z <= 32 ? 8 : 16));
     const int runs = (p->Z + k.walk - 1) / k.walk;  // walkers per column when all of Z is one chunk
 
     // super-block: as many sub-blocks as keep the whole height range in one chunk (<= 8 cells: larger
@@ -914,7 +902,8 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
     k.blocks_x = (p->X + sbx * k.wx - 1) / (sbx * k.wx);
     k.blocks_y = (p->Y + sby * k.wy - 1) / (sby * k.wy);
     k.band = 4;
-    k.reps = 1;
+    k.reps = (p->tune[3] >> 12) & 0xf;
+    if (k.reps < 1) k.reps = 1;
     k.slots = k.sbn > 1 ? 192 : 128;
     k.lcap = k.slots / k.ct;
     // height chunk: all walkers of a chunk must fit the warp's descriptor array

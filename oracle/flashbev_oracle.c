@@ -218,3 +218,107 @@ int flashbev_oracle_sampling_vt(const float *features, const float *lidar2img,
     }
     return oom ? -2 : 0;
 }
+
+
+/* ------------------------------------------------------------------------------------------
+ * Backward of the operator with respect to the features (the paper reports it in Tables 2 and 4
+ * but prints no algorithm).  The forward map is linear in the features -- masks and weights do
+ * not depend on them -- so its gradient is the transpose of that linear map, written out:
+ *
+ *   grad_features[b,n,yt,xt,c] = sum over cells, z and taps landing on (yt,xt) of
+ *                                coeff(cell,z) * w_tap * grad_out[b,ix,iy,c]
+ *   coeff = 1                                   (SUM)
+ *         = 1 / max(1, sum_z sum_n M_n)         (MEAN_OVER_VALID; the whole cell's count)
+ *         = 1 / max(1, sum_n M_n(z))            (CAMERA_MEAN_Z_SUM, Eq. 1)
+ *
+ * Plain loops in fp64; OpenMP over the (b, n) camera maps, each of which is written by one thread
+ * only (every thread re-derives the validity of all cameras for the normalisations).
+ * Pinned in tests by the adjoint identity <forward(F), G> = <F, backward(G)> against the forward
+ * oracle above, by a hand-computed sample and by structural checks.
+ */
+static int oracle_project(const float *M, double xw, double yw, double zw, double sx, double sy, int Hf, int Wf,
+                          double *fx, double *fy)
+{
+    const double p0 = (double)M[0] * xw + (double)M[1] * yw + (double)M[2] * zw + (double)M[3];
+    const double p1 = (double)M[4] * xw + (double)M[5] * yw + (double)M[6] * zw + (double)M[7];
+    const double d = (double)M[8] * xw + (double)M[9] * yw + (double)M[10] * zw + (double)M[11];
+    if (!(d > ORACLE_DEPTH_MIN)) return 0;
+    *fx = (p0 / d) * sx - 0.5;
+    *fy = (p1 / d) * sy - 0.5;
+    return (*fx > -0.5) && (*fx < (double)Wf - 0.5) && (*fy > -0.5) && (*fy < (double)Hf - 0.5);
+}
+
+/*
+ * grad_out      : host, double [B][X][Y][C]
+ * grad_features : host, double [B][N][Hf][Wf][C]   (overwritten)
+ * returns 0, or -1 on a bad argument.
+ */
+int flashbev_oracle_sampling_vt_backward(const double *grad_out, const float *lidar2img, int B, int N, int C, int Hf,
+                                         int Wf, int Himg, int Wimg, double x_min, double x_max, double y_min,
+                                         double y_max, double z_min, double z_max, int X, int Y, int Z, int reduce,
+                                         double *grad_features, int nthreads)
+{
+    if (!grad_out || !lidar2img || !grad_features) return -1;
+    if (B <= 0 || N <= 0 || C <= 0 || Hf <= 0 || Wf <= 0 || Himg <= 0 || Wimg <= 0) return -1;
+    if (X <= 0 || Y <= 0 || Z <= 0 || reduce < 0 || reduce > 2) return -1;
+    if (!(x_max > x_min) || !(y_max > y_min) || !(z_max > z_min)) return -1;
+    const double sx = (double)Wf / (double)Wimg, sy = (double)Hf / (double)Himg;
+#ifdef _OPENMP
+    if (nthreads <= 0) nthreads = omp_get_max_threads();
+#else
+    nthreads = 1;
+#endif
+#pragma omp parallel for schedule(dynamic, 1) num_threads(nthreads)
+    for (int bn = 0; bn < B * N; ++bn) {
+        const int b = bn / N, n = bn % N;
+        double *Gn = grad_features + (size_t)bn * Hf * Wf * C;
+        for (size_t i = 0; i < (size_t)Hf * Wf * C; ++i) Gn[i] = 0.0;
+        const float *Mb = lidar2img + (size_t)b * N * 16;
+        for (int ix = 0; ix < X; ++ix) {
+            for (int iy = 0; iy < Y; ++iy) {
+                const double xw = x_min + ((double)ix + 0.5) * (x_max - x_min) / (double)X;
+                const double yw = y_min + ((double)iy + 0.5) * (y_max - y_min) / (double)Y;
+                const double *go = grad_out + (((size_t)b * X + ix) * Y + iy) * C;
+                int count = 0; /* valid samples of the whole cell (MEAN_OVER_VALID) */
+                if (reduce == 1) {
+                    for (int k = 0; k < Z; ++k) {
+                        const double zw = z_min + ((double)k + 0.5) * (z_max - z_min) / (double)Z;
+                        for (int m = 0; m < N; ++m) {
+                            double fx, fy;
+                            count += oracle_project(Mb + m * 16, xw, yw, zw, sx, sy, Hf, Wf, &fx, &fy);
+                        }
+                    }
+                }
+                for (int k = 0; k < Z; ++k) {
+                    const double zw = z_min + ((double)k + 0.5) * (z_max - z_min) / (double)Z;
+                    double fx, fy;
+                    if (!oracle_project(Mb + n * 16, xw, yw, zw, sx, sy, Hf, Wf, &fx, &fy)) continue;
+                    double coeff = 1.0;
+                    if (reduce == 1) {
+                        coeff = 1.0 / (double)(count > 1 ? count : 1);
+                    } else if (reduce == 2) {
+                        int den = 0; /* cameras that see this height bin */
+                        for (int m = 0; m < N; ++m) {
+                            double gx, gy;
+                            den += oracle_project(Mb + m * 16, xw, yw, zw, sx, sy, Hf, Wf, &gx, &gy);
+                        }
+                        coeff = 1.0 / (double)(den > 1 ? den : 1);
+                    }
+                    const double x0f = floor(fx), y0f = floor(fy);
+                    const int x0 = (int)x0f, y0 = (int)y0f;
+                    const double tx = fx - x0f, ty = fy - y0f;
+                    for (int dy = 0; dy < 2; ++dy) {
+                        for (int dx = 0; dx < 2; ++dx) {
+                            const int xi = x0 + dx, yi = y0 + dy;
+                            if (xi < 0 || xi > Wf - 1 || yi < 0 || yi > Hf - 1) continue; /* zero padding */
+                            const double w = coeff * (dx ? tx : 1.0 - tx) * (dy ? ty : 1.0 - ty);
+                            double *t = Gn + ((size_t)yi * Wf + xi) * C;
+                            for (int c = 0; c < C; ++c) t[c] += w * go[c];
+                        }
+                    }
+                }
+            }
+        }
+    }
+    return 0;
+}

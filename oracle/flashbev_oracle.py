@@ -45,6 +45,8 @@ def _load():
         lib.flashbev_oracle_sampling_vt.restype = i
         lib.flashbev_oracle_sampling_vt.argtypes = (
             [p, p] + [i] * 7 + [d] * 6 + [i] * 4 + [p] * 6 + [i])
+        lib.flashbev_oracle_sampling_vt_backward.restype = i
+        lib.flashbev_oracle_sampling_vt_backward.argtypes = [p, p] + [i] * 7 + [d] * 6 + [i] * 4 + [p, i]
         lib.flashbev_oracle_max_threads.restype = i
         _lib = lib
     return _lib
@@ -93,3 +95,26 @@ def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM,
     if rc != 0:
         raise ValueError(f"flashbev_oracle_sampling_vt rejected its arguments (status {rc})")
     return OracleResult(out, count, flagged, sumw, interior.astype(bool), nzbins)
+
+
+def sampling_vt_backward(grad_out, lidar2img, feat_hw, img_hw, bev_range, grid, reduce=REDUCE_SUM, threads=0):
+    """Gradient of the operator with respect to the features (fp64).
+
+    grad_out : float64-convertible array [B, X, Y, C];  lidar2img: float32 [B, N, 4, 4]
+    Returns float64 [B, N, Hf, Wf, C].
+    """
+    g = np.ascontiguousarray(grad_out, dtype=np.float64)
+    m = np.ascontiguousarray(lidar2img, dtype=np.float32)
+    X, Y, Z = (int(v) for v in grid)
+    B, N = m.shape[:2]
+    if g.ndim != 4 or g.shape[:3] != (B, X, Y) or m.shape != (B, N, 4, 4):
+        raise ValueError("grad_out must be [B,X,Y,C] and lidar2img [B,N,4,4]")
+    C = g.shape[3]
+    Hf, Wf = (int(v) for v in feat_hw)
+    out = np.empty((B, N, Hf, Wf, C), np.float64)
+    rc = _load().flashbev_oracle_sampling_vt_backward(
+        g.ctypes.data, m.ctypes.data, B, N, C, Hf, Wf, int(img_hw[0]), int(img_hw[1]),
+        *(float(v) for v in bev_range), X, Y, Z, int(reduce), out.ctypes.data, int(threads))
+    if rc != 0:
+        raise ValueError(f"flashbev_oracle_sampling_vt_backward rejected its arguments (status {rc})")
+    return out

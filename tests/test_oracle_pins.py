@@ -356,3 +356,52 @@ def test_rejects_bad_arguments(oracle):
         oracle.sampling_vt(f, M, (4, 4), (1, -1, -1, 1, 0, 1), (1, 1, 1), SUM)   # x_max <= x_min
     with pytest.raises(ValueError):
         oracle.sampling_vt(f, M, (4, 4), (-1, 1, -1, 1, 0, 1), (1, 1, 1), 7)     # unknown reduce
+
+
+# ---------------------------------------------------------------- backward oracle (gradient w.r.t. features)
+
+@pytest.mark.parametrize("reduce", [SUM, MEAN, EQ1])
+@pytest.mark.parametrize("general", [False, True])
+def test_backward_is_the_adjoint_of_the_forward(oracle, reduce, general):
+    """<forward(F), G> == <F, backward(G)> for arbitrary F, G fixes the backward completely
+    (the forward is linear in F), so every pin of the forward oracle carries over."""
+    inp = _tiny_case(3, general, N=6, C=4, Hf=6, Wf=9, grid=(7, 6, 5))
+    w = inp.workload
+    rng = np.random.default_rng(11)
+    for trial in range(3):
+        F = rng.standard_normal(inp.features.shape).astype(np.float32)
+        G = rng.standard_normal((w.B,) + tuple(w.grid[:2]) + (w.C,))
+        out = oracle.sampling_vt(F, inp.lidar2img, w.img_hw, w.bev_range, w.grid, reduce).out
+        gF = oracle.sampling_vt_backward(G, inp.lidar2img, w.feat_hw, w.img_hw, w.bev_range, w.grid, reduce)
+        lhs, rhs = float((out * G).sum()), float((F.astype(np.float64) * gF).sum())
+        assert np.abs(out).sum() > 10.0 and np.abs(gF).sum() > 10.0      # not vacuous
+        assert lhs == pytest.approx(rhs, rel=1e-12, abs=1e-12)
+
+
+def test_backward_single_sample_by_hand(oracle):
+    # the orthographic sample of test_single_sample_orthographic_by_hand: taps (2,1) .375 (3,1) .125 (2,2) .375 (3,2) .125
+    M = ortho(1.0, 5.5, 1.0, 4.0)[None, None]
+    G = np.array([2.0, -1.0]).reshape(1, 1, 1, 2)
+    g = oracle.sampling_vt_backward(G, M, (4, 6), (8, 12), (-1, 1, -1, 1, 0, 2), (1, 1, 1), SUM)
+    expect = np.zeros((4, 6))
+    expect[1, 2], expect[1, 3], expect[2, 2], expect[2, 3] = .375, .125, .375, .125
+    assert np.allclose(g[0, 0, :, :, 0], 2.0 * expect, atol=1e-12)
+    assert np.allclose(g[0, 0, :, :, 1], -1.0 * expect, atol=1e-12)
+
+
+def test_backward_normalisations_and_untouched_texels(oracle):
+    inp = _tiny_case(4, False, N=6, C=2, Hf=6, Wf=9, grid=(7, 6, 4))
+    w = inp.workload
+    G = np.ones((w.B,) + tuple(w.grid[:2]) + (w.C,))
+    fwd = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, SUM)
+    gs = oracle.sampling_vt_backward(G, inp.lidar2img, w.feat_hw, w.img_hw, w.bev_range, w.grid, SUM)
+    gm = oracle.sampling_vt_backward(G, inp.lidar2img, w.feat_hw, w.img_hw, w.bev_range, w.grid, MEAN)
+    ge = oracle.sampling_vt_backward(G, inp.lidar2img, w.feat_hw, w.img_hw, w.bev_range, w.grid, EQ1)
+    # with G == 1 the gradient sums the weights: total mass = in-bounds weight mass of the forward
+    assert gs.sum() / w.C == pytest.approx(fwd.sumw.sum(), rel=1e-12)
+    assert np.all(gs >= 0) and np.all(gm <= gs + 1e-15) and np.all(ge <= gs + 1e-15)
+    assert (gs == 0).any()                       # texels nobody samples get exactly zero
+    # pre-scaling G by 1/max(1,count) turns the SUM backward into the MEAN backward
+    Gs = G / np.maximum(1, fwd.count)[..., None]
+    assert np.allclose(oracle.sampling_vt_backward(Gs, inp.lidar2img, w.feat_hw, w.img_hw, w.bev_range, w.grid, SUM),
+                       gm, rtol=0, atol=1e-13)

@@ -101,6 +101,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def whole_job_value(total_ms_local: float, units_per_rank: float, world: int, reduce_max=None) -> tuple:
+    """Weak-scaling aggregate: every rank processes `units_per_rank`; the job's time is the slowest
+    rank's device time.  `reduce_max(x)` returns the maximum of x over ranks (identity if None)."""
+    total_ms = float(reduce_max(total_ms_local)) if (reduce_max is not None and world > 1) else float(total_ms_local)
+    return world * units_per_rank / (total_ms * 1e-3), total_ms
+
+
 def frames_for(w: wl.Workload, min_bytes: int) -> int:
     return max(4, -(-min_bytes // w.unique_bytes))
 
@@ -232,6 +239,33 @@ def measure_workload(torch, w, args, device, rank, dist_barrier, steps, warmup, 
             "kernel": kname, "df": df}
 
 
+def measure_backward(torch, w, args, device, steps, warmup, dist_barrier):
+    """Latency of flashbev_sampling_vt_backward (memset + scatter kernel) per frame, L2-cold frames."""
+    from paper_2607_10071_b200 import binding as fb
+    X, Y, Z = w.grid
+    Hf, Wf = w.feat_hw
+    per_frame = w.output_bytes + w.B * w.N * Hf * Wf * w.C * 4
+    frames = max(4, -(-3 * L2_BYTES // per_frame))
+    base = wl.make_inputs(w)
+    mats = torch.from_numpy(base.lidar2img).to(device)
+    g = torch.Generator(device="cpu").manual_seed(99)
+    gouts = [torch.randn((w.B, X, Y, w.C), generator=g, dtype=torch.float32).to(device) for _ in range(frames)]
+    gfeats = [torch.empty((w.B, w.N, Hf, Wf, w.C), dtype=torch.float32, device=device) for _ in range(frames)]
+    ps = [fb.make_backward_params(go.data_ptr(), mats.data_ptr(), w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range,
+                                  w.grid, w.reduce, gf.data_ptr()) for go, gf in zip(gouts, gfeats)]
+    stream = torch.cuda.Stream(device)
+    with torch.cuda.stream(stream):
+        for p in ps:
+            fb.flashbev_sampling_vt_backward(p, stream.cuda_stream)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for p in ps:
+                fb.flashbev_sampling_vt_backward(p, torch.cuda.current_stream().cuda_stream)
+        total_ms, per = time_steps(torch, graph.replay, steps, warmup, dist_barrier)
+    return statistics.mean(per) / frames
+
+
 def measure_e2e(torch, w, args, device, steps, warmup, dist_barrier):
     """Same metric through flashbev_sampling_vt_host: pinned host inputs, host output, copies timed."""
     from paper_2607_10071_b200 import binding as fb
@@ -314,12 +348,13 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
 
     # max over ranks of the device time of the K steps
-    t = torch.tensor([m["total_ms"]], dtype=torch.float64, device=device)
-    if world > 1:
+    def reduce_max(x):
+        t = torch.tensor([x], dtype=torch.float64, device=device)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+        return float(t.item())
+
     frames = m["frames"]
-    value = world * args.steps * frames * w.sample_channels / (total_ms * 1e-3)
+    value, total_ms = whole_job_value(m["total_ms"], args.steps * frames * w.sample_channels, world, reduce_max)
     launch_ms = statistics.mean(m["per_step_ms"]) / frames  # average duration of one launch (one frame)
 
     # peak memory of one call: nothing may be allocated
@@ -332,10 +367,8 @@ def main():
     workspace = (torch.cuda.max_memory_allocated() - a0) + max(0, free0 - torch.cuda.mem_get_info()[0])
 
     e2e = measure_e2e(torch, w, args, device, max(3, args.steps // 4), 3, barrier)
-    te = torch.tensor([e2e["total_ms"]], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * max(3, args.steps // 4) * e2e["frames"] * w.sample_channels / (float(te.item()) * 1e-3)
+    e2e_value, _ = whole_job_value(e2e["total_ms"], max(3, args.steps // 4) * e2e["frames"] * w.sample_channels,
+                                   world, reduce_max)
 
     table = {}
     if not args.no_table and world == 1:
@@ -350,6 +383,22 @@ def main():
                            "hbm_roofline_frac_of_8TBs": wi.unique_bytes / (lat * 1e-3) / 1e9 / 8000.0,
                            "unique_mb": round(wi.unique_bytes / 1e6, 3), "output_mb": round(wi.output_bytes / 1e6, 3),
                            "kernel": mi["kernel"], "frames_per_step": mi["frames"], "reduce": wi.reduce}
+
+    context = {}
+    if not args.no_table and world == 1:
+        # the paper's own reference shape (Sec. 4.1: C=128 fp32, 56x100 maps, 200x200x8, Eq. 1), forward and
+        # backward, next to the paper's figures on its hardware -- context, not a target
+        wp = wl.get("paper_shape")
+        mf = measure_workload(torch, wp, args, device, rank, barrier, max(3, args.steps // 4), 3)
+        mf.pop("df")
+        context["paper_shape"] = {
+            "forward_latency_ms": statistics.mean(mf["per_step_ms"]) / mf["frames"],
+            "backward_latency_ms": measure_backward(torch, wp, args, device, max(3, args.steps // 4), 3, barrier),
+            "paper_forward_ms": 1.77, "paper_backward_ms": 3.27, "paper_hardware": "RTX A6000, FP32 (Table 4)",
+            "paper_trt_forward_ms": 1.128, "paper_trt_hardware": "RTX 4070 Ti SUPER, TensorRT FP32 (Table 6)"}
+        context["representative_backward_latency_ms"] = measure_backward(
+            torch, w if w.name == "representative" else wl.get("representative"), args, device,
+            max(3, args.steps // 4), 3, barrier)
 
     if rank != 0:
         if world > 1:
@@ -381,6 +430,8 @@ def main():
     }
     if table:
         line["configs"] = table
+    if context:
+        line["context"] = context
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = oracle_throughput(w, 12.0, 200)
     elif world == 1:

@@ -162,6 +162,37 @@ size_t flashbev_host_staging_bytes(const flashbev_vt_params *p); /* 0 if `p` is 
 #define FLASHBEV_STATIC_STAGING_BYTES (32u * 1024u * 1024u)
 flashbev_status flashbev_sampling_vt_host_static(const flashbev_vt_params *p, void *stream);
 
+/*
+ * Backward of the operator with respect to the features (the paper reports its cost in Tables 2
+ * and 4 without printing an algorithm).  The forward is linear in the features, so the gradient is
+ * its transpose: grad_features[b,n,y,x,c] = sum over the cells, heights and taps that read texel
+ * (y,x) of camera n of  coeff * tap weight * grad_out[b,ix,iy,c],  coeff = 1 (SUM),
+ * 1/max(1, valid samples of the cell) (MEAN_OVER_VALID), 1/max(1, cameras seeing that height bin)
+ * (CAMERA_MEAN_Z_SUM).  Geometry fields have the meaning they have in flashbev_vt_params.
+ *
+ * Enqueues on `stream` a memset of `grad_features` to zero and one kernel that scatters with
+ * fp32 vector atomics (texels are shared between cells, so the summation order -- and the last
+ * bits of the result -- can differ from run to run).  Allocates nothing.  C must be a multiple of
+ * 4 and both gradient pointers 16-byte aligned, else FLASHBEV_UNSUPPORTED / FLASHBEV_MISALIGNED.
+ */
+typedef struct flashbev_vt_backward_params {
+    size_t struct_size;        /* sizeof(flashbev_vt_backward_params) of the caller's header */
+    const float *grad_out;     /* device, [B][X][Y][C] float32; read only */
+    const float *lidar2img;    /* device, [B][N][4][4] float32; read only */
+    int32_t B, N, C;
+    int32_t feat_h, feat_w;
+    int32_t img_h, img_w;
+    double x_min, x_max;
+    double y_min, y_max;
+    double z_min, z_max;
+    int32_t X, Y, Z;
+    int32_t reduce;            /* flashbev_reduce */
+    float *grad_features;      /* device, [B][N][feat_h][feat_w][C] float32; overwritten */
+    int32_t tune[4];           /* as in flashbev_vt_params; 0 = defaults */
+} flashbev_vt_backward_params;
+
+flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params *p, void *stream);
+
 /* Number of kernels the last successful call of flashbev_sampling_vt[_host] on this thread
  * enqueued (always 1), and a short name of the kernel instance it chose (static storage). */
 int flashbev_last_launch_count(void);

@@ -46,6 +46,25 @@ class VtParams(ctypes.Structure):
     ]
 
 
+class VtBackwardParams(ctypes.Structure):
+    """Mirror of ``flashbev_vt_backward_params``."""
+    _fields_ = [
+        ("struct_size", ctypes.c_size_t),
+        ("grad_out", ctypes.c_void_p),
+        ("lidar2img", ctypes.c_void_p),
+        ("B", ctypes.c_int32), ("N", ctypes.c_int32), ("C", ctypes.c_int32),
+        ("feat_h", ctypes.c_int32), ("feat_w", ctypes.c_int32),
+        ("img_h", ctypes.c_int32), ("img_w", ctypes.c_int32),
+        ("x_min", ctypes.c_double), ("x_max", ctypes.c_double),
+        ("y_min", ctypes.c_double), ("y_max", ctypes.c_double),
+        ("z_min", ctypes.c_double), ("z_max", ctypes.c_double),
+        ("X", ctypes.c_int32), ("Y", ctypes.c_int32), ("Z", ctypes.c_int32),
+        ("reduce", ctypes.c_int32),
+        ("grad_features", ctypes.c_void_p),
+        ("tune", ctypes.c_int32 * 4),
+    ]
+
+
 class FlashBevError(RuntimeError):
     def __init__(self, status: int, what: str):
         super().__init__(f"{what}: {status_string(status)} (status {status})")
@@ -71,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.flashbev_sampling_vt_host.argtypes = [P, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         L.flashbev_sampling_vt_host_static.restype = ctypes.c_int
         L.flashbev_sampling_vt_host_static.argtypes = [P, ctypes.c_void_p]
+        L.flashbev_sampling_vt_backward.restype = ctypes.c_int
+        L.flashbev_sampling_vt_backward.argtypes = [ctypes.POINTER(VtBackwardParams), ctypes.c_void_p]
         L.flashbev_workspace_bytes.restype = ctypes.c_size_t
         L.flashbev_workspace_bytes.argtypes = [P]
         L.flashbev_host_staging_bytes.restype = ctypes.c_size_t
@@ -138,6 +159,50 @@ def flashbev_sampling_vt_host_static(params: VtParams, stream: int | None = None
     if check and st != OK:
         raise FlashBevError(st, "flashbev_sampling_vt_host_static")
     return st
+
+
+def make_backward_params(grad_out_ptr, lidar2img_ptr, B, N, C, feat_hw, img_hw, bev_range, grid, reduce,
+                         grad_features_ptr, tune=(0, 0, 0, 0)) -> VtBackwardParams:
+    p = VtBackwardParams()
+    p.struct_size = ctypes.sizeof(VtBackwardParams)
+    p.grad_out, p.lidar2img, p.grad_features = grad_out_ptr, lidar2img_ptr, grad_features_ptr
+    p.B, p.N, p.C = B, N, C
+    p.feat_h, p.feat_w = feat_hw
+    p.img_h, p.img_w = img_hw
+    p.x_min, p.x_max, p.y_min, p.y_max, p.z_min, p.z_max = (float(v) for v in bev_range)
+    p.X, p.Y, p.Z = grid
+    p.reduce = reduce
+    for i, t in enumerate(tune):
+        p.tune[i] = int(t)
+    return p
+
+
+def flashbev_sampling_vt_backward(params: VtBackwardParams, stream: int | None = None, check: bool = True) -> int:
+    """Enqueue the gradient w.r.t. the features (memset + one scatter kernel) on ``stream``."""
+    st = lib().flashbev_sampling_vt_backward(ctypes.byref(params), ctypes.c_void_p(stream or 0))
+    if check and st != OK:
+        raise FlashBevError(st, "flashbev_sampling_vt_backward")
+    return st
+
+
+def sampling_vt_backward(grad_out, lidar2img, feat_hw, img_hw, bev_range, grid, reduce=REDUCE_SUM,
+                         grad_features=None, tune=(0, 0, 0, 0), stream=None):
+    """grad_out: CUDA float32 [B,X,Y,C]; returns CUDA float32 [B,N,Hf,Wf,C] (marshalling only)."""
+    import torch
+
+    if not grad_out.is_cuda or grad_out.dtype != torch.float32 or not grad_out.is_contiguous():
+        raise ValueError("grad_out must be a contiguous CUDA float32 tensor")
+    B, X, Y, C = grad_out.shape
+    N = lidar2img.shape[1]
+    if grad_features is None:
+        grad_features = torch.empty((B, N, feat_hw[0], feat_hw[1], C), dtype=torch.float32, device=grad_out.device)
+    p = make_backward_params(grad_out.data_ptr(), lidar2img.data_ptr(), B, N, C, feat_hw, img_hw, bev_range,
+                             (X, Y, grid[2]), reduce, grad_features.data_ptr(), tune)
+    if stream is None:
+        stream = torch.cuda.current_stream(grad_out.device).cuda_stream
+    with torch.cuda.device(grad_out.device):
+        flashbev_sampling_vt_backward(p, stream)
+    return grad_features
 
 
 def flashbev_workspace_bytes(params: VtParams) -> int:

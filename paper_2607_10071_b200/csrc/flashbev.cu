@@ -35,6 +35,8 @@ struct KParams {
     const float *l2i;
     float *out;
     int32_t *count_out;
+    const float *gout;          // backward: gradient of the output [B][X][Y][C]
+    float *gfeat;               // backward: gradient of the features [B][N][Hf][Wf][C], fp32, pre-zeroed
     int B, N, C, Hf, Wf, X, Y, Z, reduce;
     double sx, sy;              // image px -> feature px
     double x_min, dx, y_min, dy, z_min, dz;
@@ -407,6 +409,56 @@ __device__ __forceinline__ bool run_walker(const KParams &p, const WarpSmem &sm,
     return true;
 }
 
+// Phase A: per (cell, camera) column of the super-block, a conservative interval of height bins of
+// the chunk [kc0, kc1) that can be valid (every validity condition is linear in z once d > 0),
+// split into walkers of at most p.walk bins.
+__device__ __forceinline__ void phase_a(const KParams &p, const WarpSmem &sm, const double *mats, const float *slope,
+                                        unsigned in_mask, int kc0, int kc1, int lane)
+{
+    for (int pr = lane; pr < p.ct * p.N; pr += 32) {
+        const int n = (pr * p.ct_inv) >> 16, c = pr - n * p.ct;
+        if (!((in_mask >> c) & 1u)) continue;
+        const double2 xy = sm.cellxy[c];
+        const double *m = mats + n * 12;
+        const float *sl = slope + n * 5;
+        const double zc0 = p.z_min + 0.5 * p.dz;  // centre of bin 0; z_w(k) = zc0 + k dz
+        // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom
+        const double d0 = fma(m[10], zc0, fma(m[9], xy.y, fma(m[8], xy.x, m[11])));
+        float lo = (float)kc0 - 1.f, hi = (float)kc1;
+        bool empty = false;
+        auto cond = [&](float a, float bslope) {
+            if (bslope > 0.f) lo = fmaxf(lo, -a * __frcp_rn(bslope));       // k > -a/b
+            else if (bslope < 0.f) hi = fminf(hi, -a * __frcp_rn(bslope));  // k < -a/b
+            else if (a <= 0.f) empty = true;  // independent of z (NaN: keep, tested exactly later)
+        };
+        cond((float)(d0 - kDepthMin), sl[0]);
+        if (empty || !(lo < hi)) continue;
+        const double p00 = fma(m[2], zc0, fma(m[1], xy.y, fma(m[0], xy.x, m[3])));
+        cond((float)p00, sl[1]);
+        cond((float)fma((double)p.Wf, d0, -p00), sl[2]);
+        if (empty || !(lo < hi)) continue;
+        const double p10 = fma(m[6], zc0, fma(m[5], xy.y, fma(m[4], xy.x, m[7])));
+        cond((float)p10, sl[3]);
+        cond((float)fma((double)p.Hf, d0, -p10), sl[4]);
+        if (empty) continue;
+        // widen by a guard far above the float error; every bin is re-tested exactly later
+        const float guard = 0.05f + 1e-5f * (float)p.Z;
+        int klo = (int)floorf(fminf(fmaxf(lo - guard, (float)kc0 - 1.f), (float)kc1)) + 1;
+        int khi = (int)ceilf(fmaxf(fminf(hi + guard, (float)kc1), (float)kc0 - 1.f)) - 1;
+        klo = max(klo, kc0);
+        khi = min(khi, kc1 - 1);
+        if (klo > khi) continue;
+        const int nw = (khi - klo + p.walk) / p.walk;
+        const int base = atomicAdd(sm.n_walkers, nw);
+        for (int i = 0; i < nw; ++i) {
+            const int k0 = klo + i * p.walk, k1 = min(khi, k0 + p.walk - 1);
+            if (base + i < p.wcap)
+                sm.walkers[base + i] = (uint32_t)c | ((uint32_t)n << 8) | ((uint32_t)(k0 - kc0) << 14) |
+                                       ((uint32_t)(k1 - k0) << 23);
+        }
+    }
+}
+
 // acc += w * (channels of one 16-byte vector), two channels per packed fp32 FMA
 template <bool BF16>
 __device__ __forceinline__ void fma_vec(float2 (&acc)[BF16 ? 4 : 2], const uint4 &t, const float2 w)
@@ -460,7 +512,25 @@ __device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], cons
     }
 }
 
-template <int V, bool BF16, int WARPS>
+// Backward of the gather: every record adds its two weighted taps of the cell's output gradient to
+// the feature gradient (the transpose of gather_list).  Vector atomics: texels are shared by cells.
+template <int V>
+__device__ __forceinline__ void scatter_list(const float4 (&go)[V], const bool (&on)[V], const int4 *list, int nrec,
+                                             float4 *const (&gfv)[V])
+{
+    for (int j = 0; j < nrec; ++j) {
+        const int4 r = list[j];
+        const float wl = __int_as_float(r.z), wr = __int_as_float(r.w);
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            if (!on[v]) continue;  // ragged last channel block
+            if (wl != 0.f) atomicAdd(gfv[v] + r.x, make_float4(go[v].x * wl, go[v].y * wl, go[v].z * wl, go[v].w * wl));
+            if (wr != 0.f) atomicAdd(gfv[v] + r.y, make_float4(go[v].x * wr, go[v].y * wr, go[v].z * wr, go[v].w * wr));
+        }
+    }
+}
+
+template <int V, bool BF16, int WARPS, bool BWD>
 __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 20 : 24)) / WARPS)
     vt_tiled_kernel(const KParams p)
 {
@@ -517,10 +587,15 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
     const int vec0 = blockIdx.y * (p.g * V) + gl;  // first channel vector of this lane
     // channel vectors past the end of the row (ragged last channel block) re-read vector 0, never stored
     const uint4 *featv[V];
+    float4 *gfv[V];  // backward: where this lane's channel vectors of a texel's gradient live
     {
-        const uint4 *featb = static_cast<const uint4 *>(p.feat) + (size_t)b * p.N * p.Hf * p.Wf * p.vecs;
+        const size_t cam0 = (size_t)b * p.N * p.Hf * p.Wf * p.vecs;
 #pragma unroll
-        for (int v = 0; v < V; ++v) featv[v] = featb + ((vec0 + v * p.g < p.vecs) ? vec0 + v * p.g : 0);
+        for (int v = 0; v < V; ++v) {
+            const int vi = (vec0 + v * p.g < p.vecs) ? vec0 + v * p.g : 0;
+            featv[v] = BWD ? nullptr : static_cast<const uint4 *>(p.feat) + cam0 + vi;
+            gfv[v] = BWD ? reinterpret_cast<float4 *>(p.gfeat) + cam0 + vi : nullptr;
+        }
     }
     const int my_tab = celltab[lane];
 
@@ -551,6 +626,31 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
             for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
         unsigned touched = 0;  // bit s: this lane has already stored its part of sub-block s
 
+        // Backward of MEAN_OVER_VALID: the cell's whole count scales every contribution, so count first.
+        if (BWD && p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) {
+            for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
+                const int kc1 = min(p.Z, kc0 + p.zc);
+                if (lane == 0) *sm.n_walkers = 0;
+                __syncwarp();
+                phase_a(p, sm, mats, slope, in_mask, kc0, kc1, lane);
+                __syncwarp();
+                const int n_walkers = min(*sm.n_walkers, p.wcap);
+                for (int wi = lane; wi < n_walkers; wi += 32) {
+                    const uint32_t wd = sm.walkers[wi];
+                    const int c = wd & 0xff, n = (wd >> 8) & 0x3f, k0 = kc0 + ((wd >> 14) & 0x1ff), k1 = k0 + (wd >> 23);
+                    ColumnWalk cw;
+                    cw.init(p, mats, n, sm.cellxy[c]);
+                    int cnt = 0;
+                    for (int k = k0; k <= k1; ++k) {
+                        Sample s;
+                        cnt += cw.sample(k, s) ? 1 : 0;
+                    }
+                    if (cnt) atomicAdd(&sm.cell_count[c], cnt);
+                }
+                __syncwarp();
+            }
+        }
+
         for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
             const int kc1 = min(p.Z, kc0 + p.zc);  // chunk [kc0, kc1)
             if (lane == 0) *sm.n_walkers = 0;
@@ -558,50 +658,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                 for (int i = lane; i < (p.ct * p.zc + 3) / 4; i += 32) sm.den[i] = 0u;
             __syncwarp();
 
-            // ---- phase A: per (cell, camera) column, a conservative interval of height bins that can
-            // be valid (every validity condition is linear in z once d > 0), split into walkers
-            for (int pr = lane; pr < p.ct * p.N; pr += 32) {
-                const int n = (pr * p.ct_inv) >> 16, c = pr - n * p.ct;
-                if (!((in_mask >> c) & 1u)) continue;
-                const double2 xy = sm.cellxy[c];
-                const double *m = mats + n * 12;
-                const float *sl = slope + n * 5;
-                const double zc0 = p.z_min + 0.5 * p.dz;  // centre of bin 0; z_w(k) = zc0 + k dz
-                // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom
-                const double d0 = fma(m[10], zc0, fma(m[9], xy.y, fma(m[8], xy.x, m[11])));
-                float lo = (float)kc0 - 1.f, hi = (float)kc1;
-                bool empty = false;
-                auto cond = [&](float a, float bslope) {
-                    if (bslope > 0.f) lo = fmaxf(lo, -a * __frcp_rn(bslope));       // k > -a/b
-                    else if (bslope < 0.f) hi = fminf(hi, -a * __frcp_rn(bslope));  // k < -a/b
-                    else if (a <= 0.f) empty = true;  // independent of z (NaN: keep, tested exactly later)
-                };
-                cond((float)(d0 - kDepthMin), sl[0]);
-                if (empty || !(lo < hi)) continue;
-                const double p00 = fma(m[2], zc0, fma(m[1], xy.y, fma(m[0], xy.x, m[3])));
-                cond((float)p00, sl[1]);
-                cond((float)fma((double)p.Wf, d0, -p00), sl[2]);
-                if (empty || !(lo < hi)) continue;
-                const double p10 = fma(m[6], zc0, fma(m[5], xy.y, fma(m[4], xy.x, m[7])));
-                cond((float)p10, sl[3]);
-                cond((float)fma((double)p.Hf, d0, -p10), sl[4]);
-                if (empty) continue;
-                // widen by a guard far above the float error; every bin is re-tested exactly later
-                const float guard = 0.05f + 1e-5f * (float)p.Z;
-                int klo = (int)floorf(fminf(fmaxf(lo - guard, (float)kc0 - 1.f), (float)kc1)) + 1;
-                int khi = (int)ceilf(fmaxf(fminf(hi + guard, (float)kc1), (float)kc0 - 1.f)) - 1;
-                klo = max(klo, kc0);
-                khi = min(khi, kc1 - 1);
-                if (klo > khi) continue;
-                const int nw = (khi - klo + p.walk) / p.walk;
-                const int base = atomicAdd(sm.n_walkers, nw);
-                for (int i = 0; i < nw; ++i) {
-                    const int k0 = klo + i * p.walk, k1 = min(khi, k0 + p.walk - 1);
-                    if (base + i < p.wcap)
-                        sm.walkers[base + i] = (uint32_t)c | ((uint32_t)n << 8) | ((uint32_t)(k0 - kc0) << 14) |
-                                               ((uint32_t)(k1 - k0) << 23);
-                }
-            }
+            phase_a(p, sm, mats, slope, in_mask, kc0, kc1, lane);
             __syncwarp();
             const int n_walkers = min(*sm.n_walkers, p.wcap);
 
@@ -654,7 +711,8 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                         w.uL = w.uR = w.lL = w.lR = 0.f;
                     }
                     if (run_walker(p, sm, mats, w, wc, wn, kend, kc0, sm.list + wc * (p.lcap + 1))) {
-                        if (w.vcount) atomicAdd(&sm.cell_count[wc], w.vcount);
+                        if (w.vcount && !(BWD && p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID))
+                            atomicAdd(&sm.cell_count[wc], w.vcount);
                     } else {
                         sm.wsave[0 * 32 + lane] = (uint32_t)w.k;
                         sm.wsave[1 * 32 + lane] = (uint32_t)w.ox;
@@ -682,6 +740,29 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                     const bool lane_on = role && ((in_mask >> cell) & 1u);
                     const int nrec = lane_on ? min(sm.list_count[cell], sm.list_end[cell]) : 0;
                     const int maxn = __reduce_max_sync(FULL, nrec);
+                    if (BWD) {
+                        if (nrec > 0) {
+                            const int tab = celltab[cell];
+                            const size_t ocell = ((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8));
+                            const int count = sm.cell_count[cell];
+                            const float gscale = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID)
+                                                     ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
+                            float4 go[V];
+                            bool on[V];
+#pragma unroll
+                            for (int v = 0; v < V; ++v) {
+                                const int vi = vec0 + v * p.g;
+                                go[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                on[v] = vi < p.vecs;
+                                if (on[v]) {
+                                    go[v] = __ldg(reinterpret_cast<const float4 *>(p.gout + ocell * p.C) + vi);
+                                    go[v].x *= gscale, go[v].y *= gscale, go[v].z *= gscale, go[v].w *= gscale;
+                                }
+                            }
+                            scatter_list<V>(go, on, sm.list + cell * (p.lcap + 1), nrec, gfv);
+                        }
+                        continue;
+                    }
                     if (p.sbn > 1) {
 #pragma unroll
                         for (int v = 0; v < V; ++v)
@@ -828,14 +909,15 @@ bool tiled_applicable(const flashbev_vt_params *p)
     return vecs_total < 2147483648.0;
 }
 
-template <int V, bool BF16, int WARPS>
+template <int V, bool BF16, int WARPS, bool BWD>
 cudaError_t launch_tiled_inst(const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
 {
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
         if (e != cudaSuccess) return e;
     }
-    vt_tiled_kernel<V, BF16, WARPS><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
+    vt_tiled_kernel<V, BF16, WARPS, BWD><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
     return cudaSuccess;
 }
 
@@ -843,22 +925,24 @@ template <int V, bool BF16>
 cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
 {
     switch (warps) {
-        case 1: return launch_tiled_inst<V, BF16, 1>(k, grid, smem, stream);
-        case 2: return launch_tiled_inst<V, BF16, 2>(k, grid, smem, stream);
-        case 8: return launch_tiled_inst<V, BF16, 8>(k, grid, smem, stream);
-        default: return launch_tiled_inst<V, BF16, 4>(k, grid, smem, stream);
+        case 1: return launch_tiled_inst<V, BF16, 1, false>(k, grid, smem, stream);
+        case 2: return launch_tiled_inst<V, BF16, 2, false>(k, grid, smem, stream);
+        case 8: return launch_tiled_inst<V, BF16, 8, false>(k, grid, smem, stream);
+        default: return launch_tiled_inst<V, BF16, 4, false>(k, grid, smem, stream);
     }
 }
 
-flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
+// Chooses the channel mapping, super-block shape, chunking and grid of the tiled kernel.
+flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V, int &warps, dim3 &grid, size_t &smem)
 {
-    KParams k = base_params(p);
+    k = base_params(p);
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     const int elem = bf16 ? 2 : 4;
     k.vecs = p->C * elem / 16;
 
     // channel mapping: V vectors per lane, g lanes per cell
-    int V = p->tune[0], g = p->tune[1];
+    V = p->tune[0];
+    int g = p->tune[1];
     if (!(V == 1 || V == 2 || V == 4) || g < 1 || g > 32) V = 0, g = 0;
     if (!V) {
         if (k.vecs <= 8) V = 1, g = k.vecs;
@@ -867,7 +951,7 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
         else V = 4, g = (k.vecs + 3) / 4;
         if (g > 32) g = 32;
     }
-    int warps = p->tune[3] & 0xf;
+    warps = p->tune[3] & 0xf;
     if (!(warps == 1 || warps == 2 || warps == 4 || warps == 8)) warps = 4;
     k.g = g;
     k.cpw = 32 / g;
@@ -921,9 +1005,21 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
     const long long ctas = (ids + (long long)warps * k.reps - 1) / ((long long)warps * k.reps);
     const int cblocks = (k.vecs + g * V - 1) / (g * V);
     if (ctas > 2147483647LL || cblocks > 65535 || p->B > 65535) return FLASHBEV_UNSUPPORTED;
-    const dim3 grid((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
-    const size_t smem = align16(cta_table_bytes(p->N)) +
+    grid = dim3((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
+    smem = align16(cta_table_bytes(p->N)) +
                         (size_t)warps * warp_smem_layout(nullptr, nullptr, k.ct, k.slots, k.zc, k.wcap);
+    return FLASHBEV_OK;
+}
+
+flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
+{
+    KParams k;
+    int V, warps;
+    dim3 grid;
+    size_t smem;
+    const flashbev_status st = configure_tiled(p, k, V, warps, grid, smem);
+    if (st != FLASHBEV_OK) return st;
+    const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     cudaError_t e;
     static const char *const names[2][3] = {{"tiled_f32_v1", "tiled_f32_v2", "tiled_f32_v4"},
                                             {"tiled_bf16_v1", "tiled_bf16_v2", "tiled_bf16_v4"}};
@@ -1026,6 +1122,54 @@ flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_s
         cudaGetLastError();
         return FLASHBEV_CUDA_ERROR;
     }
+    return FLASHBEV_OK;
+}
+
+// ---- backward --------------------------------------------------------------------------------
+flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params *q, void *stream_)
+{
+    if (!q || q->struct_size < sizeof(flashbev_vt_backward_params)) return FLASHBEV_INVALID_ARG;
+    if (!q->grad_out || !q->grad_features) return FLASHBEV_INVALID_ARG;
+    // same geometry description as the forward: validate it through the forward's checks
+    flashbev_vt_params p = {};
+    p.struct_size = sizeof(p);
+    p.features = q->grad_features;
+    p.feat_dtype = FLASHBEV_F32;
+    p.layout = FLASHBEV_NHWC;
+    p.lidar2img = q->lidar2img;
+    p.B = q->B, p.N = q->N, p.C = q->C, p.feat_h = q->feat_h, p.feat_w = q->feat_w, p.img_h = q->img_h, p.img_w = q->img_w;
+    p.x_min = q->x_min, p.x_max = q->x_max, p.y_min = q->y_min, p.y_max = q->y_max, p.z_min = q->z_min, p.z_max = q->z_max;
+    p.X = q->X, p.Y = q->Y, p.Z = q->Z, p.reduce = q->reduce;
+    p.out = const_cast<float *>(q->grad_out);
+    p.out_dtype = FLASHBEV_F32;
+    p.kernel = FLASHBEV_KERNEL_TILED;
+    for (int i = 0; i < 4; ++i) p.tune[i] = q->tune[i];
+    flashbev_status st;
+    if (!params_ok(&p, st)) return st;
+    if (((uintptr_t)q->grad_out % 16) || ((uintptr_t)q->grad_features % 16) || ((uintptr_t)q->lidar2img % 4))
+        return FLASHBEV_MISALIGNED;
+    if (q->C % 4 || !tiled_applicable(&p)) return FLASHBEV_UNSUPPORTED;
+    KParams k;
+    int V, warps;
+    dim3 grid;
+    size_t smem;
+    p.tune[3] = (p.tune[3] & ~0xf) | 4;  // the backward instances are built for 4 warps per CTA
+    if ((st = configure_tiled(&p, k, V, warps, grid, smem)) != FLASHBEV_OK) return st;
+    k.feat = nullptr, k.out = nullptr, k.count_out = nullptr;
+    k.gout = q->grad_out, k.gfeat = q->grad_features;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t bytes = (size_t)q->B * q->N * q->feat_h * q->feat_w * q->C * sizeof(float);
+    if (cudaMemsetAsync(q->grad_features, 0, bytes, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return FLASHBEV_CUDA_ERROR;
+    }
+    cudaError_t e;
+    if (V == 1) e = launch_tiled_inst<1, false, 4, true>(k, grid, smem, stream);
+    else if (V == 2) e = launch_tiled_inst<2, false, 4, true>(k, grid, smem, stream);
+    else e = launch_tiled_inst<4, false, 4, true>(k, grid, smem, stream);
+    if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+    t_last_launches = 1;
+    t_last_kernel = V == 1 ? "tiled_bwd_v1" : (V == 2 ? "tiled_bwd_v2" : "tiled_bwd_v4");
     return FLASHBEV_OK;
 }
 

@@ -41,19 +41,22 @@ def test_binding_exposes_the_same_names():
     assert fb.status_string(fb.OK) == "ok" and "unknown" in fb.status_string(99)
 
 
-def test_ctypes_struct_matches_the_c_struct(tmp_path):
+@pytest.mark.parametrize("cname,mirror", [("flashbev_vt_params", "VtParams"),
+                                          ("flashbev_vt_backward_params", "VtBackwardParams")])
+def test_ctypes_struct_matches_the_c_struct(tmp_path, cname, mirror):
     prog = tmp_path / "layout.c"
-    fields = [f[0] for f in fb.VtParams._fields_]
-    body = "\n".join(f'printf("{f} %zu\\n", offsetof(flashbev_vt_params, {f}));' for f in fields)
+    cls = getattr(fb, mirror)
+    fields = [f[0] for f in cls._fields_]
+    body = "\n".join(f'printf("{f} %zu\\n", offsetof({cname}, {f}));' for f in fields)
     prog.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "flashbev.h"\nint main(void){\n'
-                    + body + '\nprintf("sizeof %zu\\n", sizeof(flashbev_vt_params));\nreturn 0;}\n')
+                    + body + f'\nprintf("sizeof %zu\\n", sizeof({cname}));\nreturn 0;}}\n')
     exe = tmp_path / "layout"
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"), str(prog), "-o", str(exe)],
                    check=True)
     got = dict(l.split() for l in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines())
     for f in fields:
-        assert int(got[f]) == getattr(fb.VtParams, f).offset, f
-    assert int(got["sizeof"]) == ctypes.sizeof(fb.VtParams)
+        assert int(got[f]) == getattr(cls, f).offset, f
+    assert int(got["sizeof"]) == ctypes.sizeof(cls)
 
 
 def good_params(**over):

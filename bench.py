@@ -266,6 +266,28 @@ def measure_backward(torch, w, args, device, steps, warmup, dist_barrier):
     return statistics.mean(per) / frames
 
 
+def measure_tensorized(torch, w, device, iters=5):
+    """Latency and peak memory of the PyTorch tensorised baseline (paper Alg. 1) on the same GPU: context."""
+    from paper_2607_10071_b200 import tensorized_baseline as tb
+    if w.dtype != "f32":
+        return None
+    inp = wl.make_inputs(w)
+    feats = torch.from_numpy(inp.features).to(device)
+    mats = torch.from_numpy(inp.lidar2img).to(device)
+    for _ in range(2):
+        tb.sampling_vt_tensorized(feats, mats, w.img_hw, w.bev_range, w.grid, w.reduce)
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats()
+    base = torch.cuda.memory_allocated()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(iters):
+        tb.sampling_vt_tensorized(feats, mats, w.img_hw, w.bev_range, w.grid, w.reduce)
+    b.record()
+    torch.cuda.synchronize()
+    return {"latency_ms": a.elapsed_time(b) / iters, "peak_mb": (torch.cuda.max_memory_allocated() - base) / 1e6}
+
+
 def measure_e2e(torch, w, args, device, steps, warmup, dist_barrier):
     """Same metric through flashbev_sampling_vt_host: pinned host inputs, host output, copies timed."""
     from paper_2607_10071_b200 import binding as fb
@@ -396,6 +418,10 @@ def main():
             "backward_latency_ms": measure_backward(torch, wp, args, device, max(3, args.steps // 4), 3, barrier),
             "paper_forward_ms": 1.77, "paper_backward_ms": 3.27, "paper_hardware": "RTX A6000, FP32 (Table 4)",
             "paper_trt_forward_ms": 1.128, "paper_trt_hardware": "RTX 4070 Ti SUPER, TensorRT FP32 (Table 6)"}
+        context["paper_shape"]["tensorized_pytorch_baseline_on_this_gpu"] = measure_tensorized(torch, wp, device)
+        context["paper_shape"]["paper_tensorized_forward"] = {"latency_ms": 9.18, "peak_mb": 1971.94,
+                                                              "hardware": "RTX A6000 (Table 4)"}
+        context["representative_tensorized_pytorch_baseline"] = measure_tensorized(torch, wl.get("representative"), device)
         context["representative_backward_latency_ms"] = measure_backward(
             torch, w if w.name == "representative" else wl.get("representative"), args, device,
             max(3, args.steps // 4), 3, barrier)

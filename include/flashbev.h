@@ -27,8 +27,9 @@ extern "C" {
 typedef enum flashbev_status {
     FLASHBEV_OK = 0,
     FLASHBEV_INVALID_ARG = 1,  /* null pointer, non-positive size, empty range, unknown enum, short struct */
-    FLASHBEV_UNSUPPORTED = 2,  /* a combination this version does not implement (NCHW, bf16 output, sizes
-                                  beyond the 32-bit index ranges stated below) */
+    FLASHBEV_UNSUPPORTED = 2,  /* a combination this version does not implement (the tiled kernel on NCHW or
+                                  on rows that are not whole 16-byte vectors, sizes beyond the index ranges
+                                  stated below) */
     FLASHBEV_MISALIGNED = 3,   /* `out` or `lidar2img` not 4-byte aligned, `features` not element aligned */
     FLASHBEV_CUDA_ERROR = 4,   /* the launch (or a copy of the host entry point) failed; the CUDA error
                                   has been consumed with cudaGetLastError */
@@ -40,7 +41,8 @@ typedef enum flashbev_status {
 typedef enum flashbev_dtype { FLASHBEV_F32 = 0, FLASHBEV_BF16 = 1 } flashbev_dtype;
 
 /* NHWC: features [B][N][Hf][Wf][C] and out [B][X][Y][C], C contiguous (Algorithm 2 states the
- * output as B x X x Y x C).  NCHW is declared for ABI stability and returns FLASHBEV_UNSUPPORTED. */
+ * output as B x X x Y x C): the fast layout.  NCHW: features [B][N][C][Hf][Wf] and out [B][C][X][Y]
+ * (channel planes, as in Sec. 4.1); served by the per-output kernel only. */
 typedef enum flashbev_layout { FLASHBEV_NHWC = 0, FLASHBEV_NCHW = 1 } flashbev_layout;
 
 /*
@@ -99,9 +101,9 @@ typedef struct flashbev_vt_params {
     double z_min, z_max;
     int32_t X, Y, Z;           /* number of bins per axis */
     int32_t reduce;            /* flashbev_reduce */
-    void *out;                 /* [B][X][Y][C] float32; every element is written exactly once (cells no
-                                  camera sees get 0), so no pre-zeroing is needed */
-    int32_t out_dtype;         /* FLASHBEV_F32 only (bf16 output: FLASHBEV_UNSUPPORTED) */
+    void *out;                 /* [B][X][Y][C] (NHWC) or [B][C][X][Y] (NCHW), element type out_dtype; every
+                                  element is written (cells no camera sees get 0): no pre-zeroing needed */
+    int32_t out_dtype;         /* FLASHBEV_F32, or FLASHBEV_BF16: the fp32 result rounded to nearest even once */
     int32_t kernel;            /* flashbev_kernel */
     int32_t *valid_count_out;  /* optional [B][X][Y] int32: sum_z sum_n M_n per cell; NULL to skip */
     int32_t tune[4];           /* 0 = library defaults.  tune[0]: channel vectors per lane (1,2,4);

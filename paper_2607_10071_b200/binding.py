@@ -225,9 +225,11 @@ def flashbev_last_kernel_name() -> str:
 # convenience for torch callers (marshalling only)
 
 def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM, out=None,
-                valid_count=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0), stream=None):
-    """features: CUDA tensor [B,N,Hf,Wf,C] float32 or bfloat16 (contiguous); lidar2img: CUDA float32
-    [B,N,4,4].  Returns the float32 output tensor [B,X,Y,C] (allocated by torch if ``out`` is None)."""
+                valid_count=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0), stream=None, layout=NHWC,
+                out_dtype=F32):
+    """features: CUDA tensor [B,N,Hf,Wf,C] (NHWC) or [B,N,C,Hf,Wf] (NCHW), float32 or bfloat16,
+    contiguous; lidar2img: CUDA float32 [B,N,4,4].  Returns the output tensor [B,X,Y,C] (NHWC) or
+    [B,C,X,Y] (NCHW), float32 or bfloat16 per ``out_dtype`` (allocated by torch if ``out`` is None)."""
     import torch
 
     if not features.is_cuda or not lidar2img.is_cuda:
@@ -242,13 +244,17 @@ def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM,
         raise ValueError("features must be float32 or bfloat16")
     if lidar2img.dtype != torch.float32:
         raise ValueError("lidar2img must be float32")
-    B, N, Hf, Wf, C = features.shape
+    if layout == NHWC:
+        B, N, Hf, Wf, C = features.shape
+    else:
+        B, N, C, Hf, Wf = features.shape
     X, Y, Z = grid
     if out is None:
-        out = torch.empty((B, X, Y, C), dtype=torch.float32, device=features.device)
+        out = torch.empty((B, X, Y, C) if layout == NHWC else (B, C, X, Y),
+                          dtype=torch.float32 if out_dtype == F32 else torch.bfloat16, device=features.device)
     p = make_params(features.data_ptr(), dt, lidar2img.data_ptr(), B, N, C, (Hf, Wf), img_hw, bev_range,
                     (X, Y, Z), reduce, out.data_ptr(),
-                    None if valid_count is None else valid_count.data_ptr(), kernel, tune)
+                    None if valid_count is None else valid_count.data_ptr(), kernel, tune, layout, out_dtype)
     if stream is None:
         stream = torch.cuda.current_stream(features.device).cuda_stream
     with torch.cuda.device(features.device):

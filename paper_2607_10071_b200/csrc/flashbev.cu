@@ -19,6 +19,7 @@
 // Geometry (projection, validity, floor, fractions) is fp64, weights and accumulation fp32.
 #include "flashbev.h"
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -38,6 +39,7 @@ struct KParams {
     const float *gout;          // backward: gradient of the output [B][X][Y][C]
     float *gfeat;               // backward: gradient of the features [B][N][Hf][Wf][C], fp32, pre-zeroed
     int B, N, C, Hf, Wf, X, Y, Z, reduce;
+    int out_bf16;               // store the output as bfloat16 (round to nearest even) instead of float32
     double sx, sy;              // image px -> feature px
     double x_min, dx, y_min, dy, z_min, dz;
     // tiled kernel only
@@ -102,6 +104,12 @@ __device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8])
     f[5] = __uint_as_float(v.z & 0xffff0000u);
     f[6] = __uint_as_float(v.w << 16);
     f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(lo)) |
+           ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(hi)) << 16);
 }
 
 __device__ __forceinline__ float load_elem(const float *p) { return __ldg(p); }
@@ -186,16 +194,78 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
 #pragma unroll
         for (int i = 0; i < VEC; ++i) acc[i] *= g;
     }
-    float *o = p.out + (size_t)cell * p.C + c0;
-    if (VEC == 1) {
-        o[0] = acc[0];
-    } else {
+    if (p.out_bf16) {
+        uint16_t *o = reinterpret_cast<uint16_t *>(p.out) + (size_t)cell * p.C + c0;
+        if (VEC == 1) {
+            o[0] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[0]));
+        } else {
 #pragma unroll
-        for (int i = 0; i < VEC; i += 4)
-            __stcs(reinterpret_cast<float4 *>(o + i),
-                   make_float4(acc[i], acc[(i + 1) % VEC], acc[(i + 2) % VEC], acc[(i + 3) % VEC]));
+            for (int i = 0; i < VEC; i += 4)
+                *reinterpret_cast<uint2 *>(o + i) = make_uint2(pack_bf16x2(acc[i], acc[(i + 1) % VEC]),
+                                                               pack_bf16x2(acc[(i + 2) % VEC], acc[(i + 3) % VEC]));
+        }
+    } else {
+        float *o = p.out + (size_t)cell * p.C + c0;
+        if (VEC == 1) {
+            o[0] = acc[0];
+        } else {
+#pragma unroll
+            for (int i = 0; i < VEC; i += 4)
+                __stcs(reinterpret_cast<float4 *>(o + i),
+                       make_float4(acc[i], acc[(i + 1) % VEC], acc[(i + 2) % VEC], acc[(i + 3) % VEC]));
+        }
     }
     if (p.count_out && c0 == 0) p.count_out[cell] = count;
+}
+
+// Kernel 1b: the same per-output decomposition for channel-planar tensors, features
+// [B][N][C][Hf][Wf] and out [B][C][X][Y] (the layout the paper's own kernel works on, Sec. 4.1:
+// C x Hf x Wf per camera, one thread per (b, x, y, c)).  Threads are ordered with iy fastest so
+// that stores and the taps of neighbouring cells coalesce.
+template <typename T>
+__global__ void __launch_bounds__(256) vt_per_output_nchw_kernel(const KParams p)
+{
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= (long long)p.B * p.C * p.X * p.Y) return;
+    const int iy = (int)(gid % p.Y);
+    const int ix = (int)((gid / p.Y) % p.X);
+    const int c = (int)((gid / ((long long)p.X * p.Y)) % p.C);
+    const int b = (int)(gid / ((long long)p.X * p.Y * p.C));
+    const double xw = p.x_min + ((double)ix + 0.5) * p.dx;
+    const double yw = p.y_min + ((double)iy + 0.5) * p.dy;
+    const double wlim = (double)p.Wf - 0.5, hlim = (double)p.Hf - 0.5;
+    const T *feat = static_cast<const T *>(p.feat);
+    float acc = 0.f;
+    int count = 0;
+    for (int k = 0; k < p.Z; ++k) {
+        const double zw = p.z_min + ((double)k + 0.5) * p.dz;
+        float num = 0.f;
+        int den = 0;
+        for (int n = 0; n < p.N; ++n) {
+            const float *M = p.l2i + ((size_t)b * p.N + n) * 16;
+            const double p0 = fma((double)M[2], zw, fma((double)M[1], yw, fma((double)M[0], xw, (double)M[3])));
+            const double p1 = fma((double)M[6], zw, fma((double)M[5], yw, fma((double)M[4], xw, (double)M[7])));
+            const double d = fma((double)M[10], zw, fma((double)M[9], yw, fma((double)M[8], xw, (double)M[11])));
+            Sample s;
+            if (!project_sample(p0 * p.sx, p1 * p.sy, d, wlim, hlim, s)) continue;
+            den += 1;
+            const T *plane = feat + (((size_t)b * p.N + n) * p.C + c) * (size_t)p.Hf * p.Wf;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int xi = s.x0 + (t & 1), yi = s.y0 + (t >> 1);
+                if (xi < 0 || xi > p.Wf - 1 || yi < 0 || yi > p.Hf - 1) continue;  // zero padding
+                const float w = ((t & 1) ? s.tx : 1.f - s.tx) * ((t >> 1) ? s.ty : 1.f - s.ty);
+                num = fmaf(w, load_elem(plane + (size_t)yi * p.Wf + xi), num);
+            }
+        }
+        count += den;
+        if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) acc = fmaf(num, 1.f / (float)(den > 1 ? den : 1), acc);
+        else acc += num;
+    }
+    if (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) acc *= 1.f / (float)(count > 1 ? count : 1);
+    if (p.out_bf16) reinterpret_cast<uint16_t *>(p.out)[gid] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
+    else p.out[gid] = acc;
+    if (p.count_out && c == 0) p.count_out[((size_t)b * p.X + ix) * p.Y + iy] = count;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -794,8 +864,15 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                                         val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
                                     }
                                     val.x *= g, val.y *= g, val.z *= g, val.w *= g;
-                                    if (final) __stcs(dst, val);
-                                    else *dst = val;
+                                    if (p.out_bf16) {  // only with one sub-block per warp: this is the single, final store
+                                        uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C;
+                                        *reinterpret_cast<uint2 *>(ob + (size_t)vi * (PV * 2) + e * 2) =
+                                            make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
+                                    } else if (final) {
+                                        __stcs(dst, val);
+                                    } else {
+                                        *dst = val;
+                                    }
                                 }
                             }
                         }
@@ -837,7 +914,7 @@ bool params_ok(const flashbev_vt_params *p, flashbev_status &st)
     if (p->out_dtype != FLASHBEV_F32 && p->out_dtype != FLASHBEV_BF16) return false;
     if (p->kernel < 0 || p->kernel > 2) return false;
     st = FLASHBEV_UNSUPPORTED;
-    if (p->layout != FLASHBEV_NHWC || p->out_dtype != FLASHBEV_F32) return false;
+    if (p->layout == FLASHBEV_NCHW && p->kernel == FLASHBEV_KERNEL_TILED) return false;  // planar: per-output kernel only
     if (p->N > kMaxCams) return false;
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
     const double cam_bytes = (double)p->N * p->feat_h * p->feat_w * p->C * (double)elem;
@@ -851,7 +928,8 @@ bool params_ok(const flashbev_vt_params *p, flashbev_status &st)
 flashbev_status check_alignment(const flashbev_vt_params *p)
 {
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
-    if (((uintptr_t)p->features % elem) || ((uintptr_t)p->out % 4) || ((uintptr_t)p->lidar2img % 4)) return FLASHBEV_MISALIGNED;
+    const size_t oelem = p->out_dtype == FLASHBEV_F32 ? 4 : 2;
+    if (((uintptr_t)p->features % elem) || ((uintptr_t)p->out % oelem) || ((uintptr_t)p->lidar2img % 4)) return FLASHBEV_MISALIGNED;
     if (p->valid_count_out && ((uintptr_t)p->valid_count_out % 4)) return FLASHBEV_MISALIGNED;
     return FLASHBEV_OK;
 }
@@ -865,6 +943,7 @@ KParams base_params(const flashbev_vt_params *p)
     k.count_out = p->valid_count_out;
     k.B = p->B, k.N = p->N, k.C = p->C, k.Hf = p->feat_h, k.Wf = p->feat_w;
     k.X = p->X, k.Y = p->Y, k.Z = p->Z, k.reduce = p->reduce;
+    k.out_bf16 = p->out_dtype == FLASHBEV_BF16;
     k.sx = (double)p->feat_w / (double)p->img_w;
     k.sy = (double)p->feat_h / (double)p->img_h;
     k.x_min = p->x_min, k.dx = (p->x_max - p->x_min) / (double)p->X;
@@ -877,6 +956,15 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
 {
     const KParams k = base_params(p);
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
+    if (p->layout == FLASHBEV_NCHW) {
+        const long long threads = (long long)p->B * p->C * p->X * p->Y;
+        const long long blocks = (threads + 255) / 256;
+        if (blocks > 2147483647LL) return FLASHBEV_UNSUPPORTED;
+        if (bf16) vt_per_output_nchw_kernel<uint16_t><<<dim3((unsigned)blocks), dim3(256), 0, stream>>>(k);
+        else vt_per_output_nchw_kernel<float><<<dim3((unsigned)blocks), dim3(256), 0, stream>>>(k);
+        t_last_kernel = bf16 ? "per_output_nchw_bf16" : "per_output_nchw_f32";
+        return FLASHBEV_OK;
+    }
     const int vec = bf16 ? 8 : 4;
     const bool vec_ok = (p->C % vec == 0) && ((uintptr_t)p->features % 16 == 0) && ((uintptr_t)p->out % 16 == 0);
     const int per_thread = vec_ok ? vec : 1;
@@ -902,6 +990,7 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
 
 bool tiled_applicable(const flashbev_vt_params *p)
 {
+    if (p->layout != FLASHBEV_NHWC) return false;
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
     if (((size_t)p->C * elem) % 16) return false;
     if (((uintptr_t)p->features % 16) || ((uintptr_t)p->out % 16)) return false;
@@ -969,7 +1058,9 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     // super-block: as many sub-blocks as keep the whole height range in one chunk (<= 8 cells: larger
     // ones pack the geometry lanes better but leave too few warps to overlap geometry with gathers)
     int sbx = (p->tune[3] >> 4) & 0xf, sby = (p->tune[3] >> 8) & 0xf;
-    if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
+    if (k.out_bf16) {
+        sbx = sby = 1;  // a rounded output cannot take partial sums: keep the accumulators in registers
+    } else if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
         sbx = sby = 1;
         while (true) {
             const bool grow_x = sbx * k.wx <= sby * k.wy;
@@ -1060,7 +1151,7 @@ StagingLayout staging_layout(const flashbev_vt_params *p)
     s.feat_off = 0;
     s.mat_off = up((size_t)p->B * p->N * p->feat_h * p->feat_w * p->C * elem);
     s.out_off = s.mat_off + up((size_t)p->B * p->N * 64);
-    s.cnt_off = s.out_off + up((size_t)p->B * p->X * p->Y * p->C * 4);
+    s.cnt_off = s.out_off + up((size_t)p->B * p->X * p->Y * p->C * (p->out_dtype == FLASHBEV_F32 ? 4 : 2));
     s.total = s.cnt_off + (p->valid_count_out ? up((size_t)p->B * p->X * p->Y * 4) : 0);
     return s;
 }
@@ -1115,7 +1206,8 @@ flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_s
         return FLASHBEV_CUDA_ERROR;
     }
     if ((st = run_device(&d, stream)) != FLASHBEV_OK) return st;
-    if (cudaMemcpyAsync(p->out, base + L.out_off, (size_t)p->B * p->X * p->Y * p->C * 4, cudaMemcpyDeviceToHost, stream) !=
+    if (cudaMemcpyAsync(p->out, base + L.out_off, (size_t)p->B * p->X * p->Y * p->C * (p->out_dtype == FLASHBEV_F32 ? 4 : 2),
+                        cudaMemcpyDeviceToHost, stream) !=
             cudaSuccess ||
         (p->valid_count_out && cudaMemcpyAsync(p->valid_count_out, base + L.cnt_off, (size_t)p->B * p->X * p->Y * 4,
                                                cudaMemcpyDeviceToHost, stream) != cudaSuccess)) {

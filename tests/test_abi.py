@@ -79,8 +79,8 @@ def good_params(**over):
     (dict(bev_range=(-25, float("inf"), -25, 25, -3, 1)), fb.INVALID_ARG),
     (dict(reduce=3), fb.INVALID_ARG), (dict(feat_dtype=2), fb.INVALID_ARG), (dict(kernel=9), fb.INVALID_ARG),
     (dict(layout=7), fb.INVALID_ARG),
-    (dict(layout=fb.NCHW), fb.UNSUPPORTED),
-    (dict(out_dtype=fb.BF16), fb.UNSUPPORTED),
+    (dict(layout=fb.NCHW, kernel=fb.KERNEL_TILED), fb.UNSUPPORTED),  # planar tensors: per-output kernel only
+    (dict(out_dtype=fb.BF16, out_ptr=16385), fb.MISALIGNED),
     (dict(N=65), fb.UNSUPPORTED),
     (dict(B=1 << 20, grid=(1 << 10, 1 << 10, 4)), fb.UNSUPPORTED),
     (dict(features_ptr=4098), fb.MISALIGNED),

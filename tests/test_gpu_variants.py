@@ -1,0 +1,90 @@
+"""Variants of the operator: channel-planar (NCHW) tensors and bfloat16 output."""
+import numpy as np
+import pytest
+
+from paper_2607_10071_b200 import binding as fb
+from paper_2607_10071_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+SUM, MEAN, EQ1 = 0, 1, 2
+
+
+def _cuda_features(inp, layout):
+    import torch
+    w = inp.workload
+    dev = torch.device("cuda:0")
+    if w.dtype == "bf16":
+        f = torch.from_numpy(inp.features_bf16.view(np.int16)).to(dev).view(torch.bfloat16)
+    else:
+        f = torch.from_numpy(inp.features).to(dev)
+    if layout == fb.NCHW:
+        f = f.permute(0, 1, 4, 2, 3).contiguous()
+    return f, torch.from_numpy(inp.lidar2img).to(dev)
+
+
+def _bf16_to_f32(t):
+    import torch
+    return t.to(torch.float32).cpu().numpy()
+
+
+@pytest.mark.parametrize("reduce", [SUM, MEAN, EQ1])
+@pytest.mark.parametrize("dtype,C", [("f32", 5), ("f32", 32), ("bf16", 24), ("bf16", 7)])
+def test_nchw_tensors(oracle, reduce, dtype, C):
+    import torch
+    w = wl.Workload(f"nchw{C}", 3000 + C, 2, 5, C, dtype, (10, 14), (80, 112), (17, 13, 6),
+                    (-10.0, 10.0, -10.0, 10.0, -3.0, 2.0), 0, general_pose=True)
+    inp = wl.make_inputs(w)
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, reduce)
+    f, m = _cuda_features(inp, fb.NCHW)
+    X, Y, Z = w.grid
+    cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=f.device)
+    out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, valid_count=cnt, layout=fb.NCHW)
+    assert fb.flashbev_last_kernel_name().startswith("per_output_nchw")
+    assert out.shape == (w.B, C, X, Y)
+    parity.assert_parity(w, ref, out.permute(0, 2, 3, 1).cpu().numpy(), cnt.cpu().numpy(), "[nchw]", check_fraction=False)
+
+
+def test_nchw_benchmark_shape(oracle):
+    import torch
+    w = wl.get("tiny")
+    inp = wl.make_inputs(w)
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, EQ1)
+    f, m = _cuda_features(inp, fb.NCHW)
+    out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, EQ1, layout=fb.NCHW)
+    parity.assert_parity(w, ref, out.permute(0, 2, 3, 1).cpu().numpy(), None, "[nchw tiny]")
+
+
+@pytest.mark.parametrize("kernel", [fb.KERNEL_AUTO, fb.KERNEL_PER_OUTPUT])
+@pytest.mark.parametrize("name,reduce", [("tiny", SUM), ("representative", EQ1), ("half_taller", MEAN)])
+def test_bf16_output_is_the_fp32_result_rounded_once(oracle, kernel, name, reduce):
+    """|out - oracle| <= (tolerance of the fp32-output path) + half a bf16 ulp of the value (2^-9 |ref|)."""
+    import torch
+    w = wl.get(name)
+    inp = wl.make_inputs(w)
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, reduce)
+    f, m = _cuda_features(inp, fb.NHWC)
+    out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, kernel=kernel, out_dtype=fb.BF16)
+    assert out.dtype == torch.bfloat16
+    got = _bf16_to_f32(out).astype(np.float64)
+    keep = ref.flagged == 0
+    base = 1e-4 if w.dtype == "f32" else 2e-3 * np.sqrt(np.maximum(1, ref.count))[..., None]
+    bound = (base + np.abs(ref.out) * 2.0 ** -8 + 1e-30) * np.ones_like(ref.out)
+    err = np.abs(got - ref.out)
+    assert np.all(err[keep] <= bound[keep]), float((err / bound)[keep].max())
+    # and it is exactly the rounding of the fp32 output of the same kernel
+    out32 = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, kernel=kernel)
+    if kernel == fb.KERNEL_PER_OUTPUT:
+        assert torch.equal(out32.to(torch.bfloat16), out)
+
+
+def test_bf16_output_with_nchw(oracle):
+    import torch
+    w = wl.Workload("nchw_bf16out", 3100, 1, 4, 6, "f32", (8, 12), (64, 96), (9, 8, 4),
+                    (-8.0, 8.0, -8.0, 8.0, -3.0, 2.0), 0, general_pose=True)
+    inp = wl.make_inputs(w)
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, SUM)
+    f, m = _cuda_features(inp, fb.NCHW)
+    out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, SUM, layout=fb.NCHW, out_dtype=fb.BF16)
+    got = _bf16_to_f32(out.permute(0, 2, 3, 1)).astype(np.float64)
+    assert np.all(np.abs(got - ref.out) <= 1e-4 + np.abs(ref.out) * 2.0 ** -8)

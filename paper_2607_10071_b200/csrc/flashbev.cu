@@ -988,6 +988,26 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
     return FLASHBEV_OK;
 }
 
+// Number of SMs of the current device (cached per device; 148 on a B200).
+int sm_count()
+{
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return 148;
+    }
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = 148;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 bool tiled_applicable(const flashbev_vt_params *p)
 {
     if (p->layout != FLASHBEV_NHWC) return false;
@@ -1068,6 +1088,8 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
             const int ct = nx * ny * k.cpw;
             // keep the whole height range in one chunk and leave each cell a list of ~1.5 Z + 4 records
             if (ct > 8 || (long long)ct * p->N * runs > 512 || 2 * ct * (3 * p->Z + 8) > 2 * 2 * 192) break;
+            // small problems: rather one warp per sub-block than idle SMs (a warp's latency is the kernel's)
+            if ((long long)p->B * p->X * p->Y / ct < (long long)sm_count() * 24) break;
             sbx = nx, sby = ny;
         }
     }

@@ -405,3 +405,17 @@ def test_backward_normalisations_and_untouched_texels(oracle):
     Gs = G / np.maximum(1, fwd.count)[..., None]
     assert np.allclose(oracle.sampling_vt_backward(Gs, inp.lidar2img, w.feat_hw, w.img_hw, w.bev_range, w.grid, SUM),
                        gm, rtol=0, atol=1e-13)
+
+
+def test_oracle_has_not_drifted_from_its_committed_outputs(oracle):
+    """Regression guard (not a correctness pin): values written by tests/golden/make_oracle_regression.py."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_oracle_regression", os.path.join(GOLDEN, "make_oracle_regression.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    want = [l.split() for l in open(os.path.join(GOLDEN, "oracle_regression.txt")) if not l.startswith("#")]
+    got = mod.rows()
+    assert len(want) == len(got) == 15
+    for wrow, grow in zip(want, got):
+        assert [int(v) for v in wrow[:5]] == list(grow[:5])
+        assert float(wrow[5]) == pytest.approx(grow[5], rel=1e-13, abs=1e-13)

@@ -322,3 +322,124 @@ int flashbev_oracle_sampling_vt_backward(const double *grad_out, const float *li
     }
     return 0;
 }
+
+
+/* ------------------------------------------------------------------------------------------
+ * FlashSCA: spatial cross-attention with on-the-fly projection (paper Sec. 4.4, "Cross-framework
+ * applicability").  The paper states the idea only; the operator is the deformable-attention view
+ * transformation of BEVFormer, restated here:
+ *
+ *   every BEV query q = (ix, iy) owns Zref reference heights (bin centres of [z_min, z_max]);
+ *   reference k is projected into camera n exactly as in the Sampling-VT operator; it is VALID iff
+ *   depth > 0.1 and the pixel lies strictly inside the image; (ru, rv) = (u / Wimg, v / Himg);
+ *   camera n is HIT by q iff at least one of its references is valid;
+ *   for every hit camera, head h, level l and point p (which uses reference k = p mod Zref):
+ *       pixel position in level l:  px = ru W_l + dx - 1/2,  py = rv H_l + dy - 1/2
+ *       ((dx, dy) = offsets[b,q,h,l,p], in texels of level l; align_corners = False),
+ *       s = bilinear sample of value level l of camera n, channels of head h, zero padding,
+ *       and the point contributes  A[b,q,h,l,p] * s  if its reference is valid (this reading
+ *       masks per reference; the original masks per camera only);
+ *   out[b,q,h,:] = (sum over hit cameras, levels, points) / max(1, number of hit cameras).
+ *
+ * value   : host float32 [B][N][T][heads*Dh], T = sum_l H_l W_l texels, levels concatenated
+ * level_hw: host int32 [L][2] = (H_l, W_l)
+ * offsets : host float32 [B][Q][heads][L][P][2];  weights: host float32 [B][Q][heads][L][P]
+ * out     : host double [B][Q][heads*Dh];  hits / flagged: host int32 [B][Q] (may be NULL)
+ * Q = X*Y with q = ix*Y + iy.  Returns 0, or -1 on a bad argument.
+ */
+int flashbev_oracle_sca(const float *value, const int32_t *level_hw, const float *lidar2img, const float *offsets,
+                        const float *weights, int B, int N, int heads, int Dh, int L, int P, int Himg, int Wimg,
+                        double x_min, double x_max, double y_min, double y_max, double z_min, double z_max, int X,
+                        int Y, int Zref, double *out, int32_t *hits, int32_t *flagged, int nthreads)
+{
+    if (!value || !level_hw || !lidar2img || !offsets || !weights || !out) return -1;
+    if (B <= 0 || N <= 0 || heads <= 0 || Dh <= 0 || L <= 0 || P <= 0 || Himg <= 0 || Wimg <= 0) return -1;
+    if (X <= 0 || Y <= 0 || Zref <= 0 || N > 64 || Zref > 64) return -1;
+    if (!(x_max > x_min) || !(y_max > y_min) || !(z_max > z_min)) return -1;
+    const int D = heads * Dh, Q = X * Y;
+    long long T = 0;
+    for (int l = 0; l < L; ++l) {
+        if (level_hw[2 * l] <= 0 || level_hw[2 * l + 1] <= 0) return -1;
+        T += (long long)level_hw[2 * l] * level_hw[2 * l + 1];
+    }
+#ifdef _OPENMP
+    if (nthreads <= 0) nthreads = omp_get_max_threads();
+#else
+    nthreads = 1;
+#endif
+#pragma omp parallel for schedule(dynamic, 16) num_threads(nthreads)
+    for (long long bq = 0; bq < (long long)B * Q; ++bq) {
+        const int b = (int)(bq / Q), q = (int)(bq % Q);
+        const int ix = q / Y, iy = q % Y;
+        const double xw = x_min + ((double)ix + 0.5) * (x_max - x_min) / (double)X;
+        const double yw = y_min + ((double)iy + 0.5) * (y_max - y_min) / (double)Y;
+        double ru[64][64], rv[64][64]; /* [n][k] */
+        int valid[64][64], hit[64], nhit = 0, flg = 0;
+        for (int n = 0; n < N; ++n) {
+            const float *M = lidar2img + ((size_t)b * N + n) * 16;
+            hit[n] = 0;
+            for (int k = 0; k < Zref; ++k) {
+                const double zw = z_min + ((double)k + 0.5) * (z_max - z_min) / (double)Zref;
+                const double p0 = (double)M[0] * xw + (double)M[1] * yw + (double)M[2] * zw + (double)M[3];
+                const double p1 = (double)M[4] * xw + (double)M[5] * yw + (double)M[6] * zw + (double)M[7];
+                const double d = (double)M[8] * xw + (double)M[9] * yw + (double)M[10] * zw + (double)M[11];
+                valid[n][k] = 0;
+                ru[n][k] = rv[n][k] = 0.0;
+                if (!(d > ORACLE_DEPTH_MIN - ORACLE_BORDER_EPS)) continue;
+                const double u = p0 / d, v = p1 / d;
+                if (isfinite(u) && isfinite(v)) { /* smallest signed margin: image px, depth m */
+                    double m = d - ORACLE_DEPTH_MIN;
+                    if (u < m) m = u;
+                    if ((double)Wimg - u < m) m = (double)Wimg - u;
+                    if (v < m) m = v;
+                    if ((double)Himg - v < m) m = (double)Himg - v;
+                    if (fabs(m) < ORACLE_BORDER_EPS) flg += 1;
+                }
+                if (d > ORACLE_DEPTH_MIN && u > 0.0 && u < (double)Wimg && v > 0.0 && v < (double)Himg) {
+                    valid[n][k] = 1;
+                    ru[n][k] = u / (double)Wimg;
+                    rv[n][k] = v / (double)Himg;
+                    hit[n] = 1;
+                }
+            }
+            nhit += hit[n];
+        }
+        double *o = out + (size_t)bq * D;
+        for (int c = 0; c < D; ++c) o[c] = 0.0;
+        for (int n = 0; n < N; ++n) {
+            if (!hit[n]) continue;
+            const float *Vn = value + ((size_t)b * N + n) * (size_t)T * D;
+            for (int h = 0; h < heads; ++h) {
+                long long lvl0 = 0;
+                for (int l = 0; l < L; ++l) {
+                    const int Hl = level_hw[2 * l], Wl = level_hw[2 * l + 1];
+                    for (int p = 0; p < P; ++p) {
+                        const int k = p % Zref;
+                        if (!valid[n][k]) continue;
+                        const size_t sidx = ((((size_t)b * Q + q) * heads + h) * L + l) * P + p;
+                        const double A = (double)weights[sidx];
+                        const double px = ru[n][k] * (double)Wl + (double)offsets[2 * sidx] - 0.5;
+                        const double py = rv[n][k] * (double)Hl + (double)offsets[2 * sidx + 1] - 0.5;
+                        const double x0f = floor(px), y0f = floor(py);
+                        const double tx = px - x0f, ty = py - y0f;
+                        for (int dy = 0; dy < 2; ++dy) {
+                            for (int dx = 0; dx < 2; ++dx) {
+                                const double xi = x0f + dx, yi = y0f + dy;
+                                if (!(xi >= 0.0 && xi <= (double)(Wl - 1) && yi >= 0.0 && yi <= (double)(Hl - 1))) continue;
+                                const double w = A * (dx ? tx : 1.0 - tx) * (dy ? ty : 1.0 - ty);
+                                const float *t = Vn + ((size_t)lvl0 + (size_t)yi * Wl + (size_t)xi) * D + (size_t)h * Dh;
+                                for (int e = 0; e < Dh; ++e) o[h * Dh + e] += w * (double)t[e];
+                            }
+                        }
+                    }
+                    lvl0 += (long long)Hl * Wl;
+                }
+            }
+        }
+        const double g = 1.0 / (double)(nhit > 1 ? nhit : 1);
+        for (int c = 0; c < D; ++c) o[c] *= g;
+        if (hits) hits[bq] = nhit;
+        if (flagged) flagged[bq] = flg;
+    }
+    return 0;
+}

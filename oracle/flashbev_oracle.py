@@ -47,6 +47,8 @@ def _load():
             [p, p] + [i] * 7 + [d] * 6 + [i] * 4 + [p] * 6 + [i])
         lib.flashbev_oracle_sampling_vt_backward.restype = i
         lib.flashbev_oracle_sampling_vt_backward.argtypes = [p, p] + [i] * 7 + [d] * 6 + [i] * 4 + [p, i]
+        lib.flashbev_oracle_sca.restype = i
+        lib.flashbev_oracle_sca.argtypes = [p] * 5 + [i] * 8 + [d] * 6 + [i] * 3 + [p] * 3 + [i]
         lib.flashbev_oracle_max_threads.restype = i
         _lib = lib
     return _lib
@@ -118,3 +120,35 @@ def sampling_vt_backward(grad_out, lidar2img, feat_hw, img_hw, bev_range, grid, 
     if rc != 0:
         raise ValueError(f"flashbev_oracle_sampling_vt_backward rejected its arguments (status {rc})")
     return out
+
+
+def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, threads=0):
+    """Spatial cross-attention with on-the-fly projection (fp64).
+
+    value   : float32 [B, N, T, heads, Dh]   (T = sum of H_l * W_l, levels concatenated)
+    level_hw: int [L, 2];  lidar2img: float32 [B, N, 4, 4]
+    offsets : float32 [B, Q, heads, L, P, 2] (texels of the level);  weights: float32 [B, Q, heads, L, P]
+    grid    : (X, Y, Zref), Q = X * Y.   Returns (out float64 [B, Q, heads*Dh], hits int32 [B, Q], flagged int32 [B, Q]).
+    """
+    v = np.ascontiguousarray(value, np.float32)
+    lv = np.ascontiguousarray(level_hw, np.int32)
+    m = np.ascontiguousarray(lidar2img, np.float32)
+    of = np.ascontiguousarray(offsets, np.float32)
+    wt = np.ascontiguousarray(weights, np.float32)
+    B, N, T, heads, Dh = v.shape
+    X, Y, Zref = (int(t) for t in grid)
+    Q = X * Y
+    L, P = wt.shape[3], wt.shape[4]
+    if lv.shape != (L, 2) or int((lv[:, 0] * lv[:, 1]).sum()) != T or of.shape != (B, Q, heads, L, P, 2) \
+            or wt.shape != (B, Q, heads, L, P) or m.shape != (B, N, 4, 4):
+        raise ValueError("inconsistent shapes")
+    out = np.empty((B, Q, heads * Dh), np.float64)
+    hits = np.empty((B, Q), np.int32)
+    flagged = np.empty((B, Q), np.int32)
+    rc = _load().flashbev_oracle_sca(
+        v.ctypes.data, lv.ctypes.data, m.ctypes.data, of.ctypes.data, wt.ctypes.data, B, N, heads, Dh, L, P,
+        int(img_hw[0]), int(img_hw[1]), *(float(t) for t in bev_range), X, Y, Zref,
+        out.ctypes.data, hits.ctypes.data, flagged.ctypes.data, int(threads))
+    if rc != 0:
+        raise ValueError(f"flashbev_oracle_sca rejected its arguments (status {rc})")
+    return out, hits, flagged

@@ -195,6 +195,44 @@ typedef struct flashbev_vt_backward_params {
 
 flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params *p, void *stream);
 
+/*
+ * FlashSCA: spatial cross-attention with on-the-fly projection (Sec. 4.4, "Cross-framework
+ * applicability"; the paper states the idea, the operator is BEVFormer's deformable-attention view
+ * transformation).  Every BEV query q = (ix, iy) has Zref reference heights (bin centres of
+ * [z_min, z_max]); reference k is projected into camera n with lidar2img exactly as in
+ * flashbev_vt_params and is valid iff depth > 0.1 and the pixel is strictly inside the image.  A
+ * camera is hit by the query iff one of its references is valid.  For every hit camera, head h,
+ * level l and sampling point p (which uses reference k = p mod Zref, if valid) the value map is
+ * sampled bilinearly (align_corners=False, zero padding) at
+ *     px = u / img_w * W_l + offsets[..][0] - 1/2,   py = v / img_h * H_l + offsets[..][1] - 1/2
+ * and out[b][q][h][:] = sum(weights * sample) / max(1, number of hit cameras).
+ * References are projected in fp64, interpolation weights and accumulation are fp32.  One kernel on
+ * `stream`; nothing allocated; no per-camera BEV-shaped intermediate is ever stored.
+ */
+typedef struct flashbev_sca_params {
+    size_t struct_size;        /* sizeof(flashbev_sca_params) of the caller's header */
+    const void *value;         /* device, [B][N][T][heads][head_dim], T = sum_l H_l*W_l (levels concatenated,
+                                  each level row-major); value_dtype, 16-byte aligned */
+    int32_t value_dtype;       /* FLASHBEV_F32 (bf16 values: FLASHBEV_UNSUPPORTED) */
+    int32_t reserved;
+    const int32_t *level_hw;   /* HOST, [L][2] = (H_l, W_l); read during the call only; L <= 8 */
+    const float *lidar2img;    /* device, [B][N][4][4] float32 */
+    const float *offsets;      /* device, [B][X*Y][heads][L][P][2] float32, in texels of level l */
+    const float *weights;      /* device, [B][X*Y][heads][L][P] float32 (normally a softmax over L*P) */
+    int32_t B, N, heads, head_dim; /* head_dim a multiple of 4, <= 128; heads * head_dim / 4 <= 128 lanes x 4 */
+    int32_t L, P;
+    int32_t img_h, img_w;
+    double x_min, x_max;
+    double y_min, y_max;
+    double z_min, z_max;
+    int32_t X, Y, Zref;        /* queries q = ix * Y + iy; Zref <= 32 */
+    int32_t reserved2;
+    float *out;                /* device, [B][X*Y][heads*head_dim] float32; every element written */
+    int32_t *hits_out;         /* optional device [B][X*Y] int32: cameras that see the query */
+} flashbev_sca_params;
+
+flashbev_status flashbev_sca(const flashbev_sca_params *p, void *stream);
+
 /* Number of kernels the last successful call of flashbev_sampling_vt[_host] on this thread
  * enqueued (always 1), and a short name of the kernel instance it chose (static storage). */
 int flashbev_last_launch_count(void);

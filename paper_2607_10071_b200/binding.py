@@ -65,6 +65,28 @@ class VtBackwardParams(ctypes.Structure):
     ]
 
 
+class ScaParams(ctypes.Structure):
+    """Mirror of ``flashbev_sca_params``."""
+    _fields_ = [
+        ("struct_size", ctypes.c_size_t),
+        ("value", ctypes.c_void_p),
+        ("value_dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("level_hw", ctypes.c_void_p),
+        ("lidar2img", ctypes.c_void_p),
+        ("offsets", ctypes.c_void_p),
+        ("weights", ctypes.c_void_p),
+        ("B", ctypes.c_int32), ("N", ctypes.c_int32), ("heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("L", ctypes.c_int32), ("P", ctypes.c_int32),
+        ("img_h", ctypes.c_int32), ("img_w", ctypes.c_int32),
+        ("x_min", ctypes.c_double), ("x_max", ctypes.c_double),
+        ("y_min", ctypes.c_double), ("y_max", ctypes.c_double),
+        ("z_min", ctypes.c_double), ("z_max", ctypes.c_double),
+        ("X", ctypes.c_int32), ("Y", ctypes.c_int32), ("Zref", ctypes.c_int32), ("reserved2", ctypes.c_int32),
+        ("out", ctypes.c_void_p),
+        ("hits_out", ctypes.c_void_p),
+    ]
+
+
 class FlashBevError(RuntimeError):
     def __init__(self, status: int, what: str):
         super().__init__(f"{what}: {status_string(status)} (status {status})")
@@ -92,6 +114,8 @@ def lib() -> ctypes.CDLL:
         L.flashbev_sampling_vt_host_static.argtypes = [P, ctypes.c_void_p]
         L.flashbev_sampling_vt_backward.restype = ctypes.c_int
         L.flashbev_sampling_vt_backward.argtypes = [ctypes.POINTER(VtBackwardParams), ctypes.c_void_p]
+        L.flashbev_sca.restype = ctypes.c_int
+        L.flashbev_sca.argtypes = [ctypes.POINTER(ScaParams), ctypes.c_void_p]
         L.flashbev_workspace_bytes.restype = ctypes.c_size_t
         L.flashbev_workspace_bytes.argtypes = [P]
         L.flashbev_host_staging_bytes.restype = ctypes.c_size_t
@@ -203,6 +227,47 @@ def sampling_vt_backward(grad_out, lidar2img, feat_hw, img_hw, bev_range, grid, 
     with torch.cuda.device(grad_out.device):
         flashbev_sampling_vt_backward(p, stream)
     return grad_features
+
+
+def flashbev_sca(params: ScaParams, stream: int | None = None, check: bool = True) -> int:
+    """Enqueue the fused spatial cross-attention on ``stream``."""
+    st = lib().flashbev_sca(ctypes.byref(params), ctypes.c_void_p(stream or 0))
+    if check and st != OK:
+        raise FlashBevError(st, "flashbev_sca")
+    return st
+
+
+def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, out=None, hits=None, stream=None):
+    """value: CUDA float32 [B,N,T,heads,Dh]; offsets [B,Q,heads,L,P,2]; weights [B,Q,heads,L,P] (CUDA float32).
+    level_hw: sequence of (H_l, W_l).  Returns CUDA float32 [B, Q, heads*Dh] (marshalling only)."""
+    import numpy as np
+    import torch
+
+    for t in (value, lidar2img, offsets, weights):
+        if not t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError("sca needs contiguous CUDA float32 tensors")
+    B, N, T, heads, Dh = value.shape
+    X, Y, Zref = grid
+    L, P = weights.shape[3], weights.shape[4]
+    lv = np.ascontiguousarray(level_hw, np.int32)
+    if out is None:
+        out = torch.empty((B, X * Y, heads * Dh), dtype=torch.float32, device=value.device)
+    p = ScaParams()
+    p.struct_size = ctypes.sizeof(ScaParams)
+    p.value, p.value_dtype = value.data_ptr(), F32
+    p.level_hw = lv.ctypes.data
+    p.lidar2img, p.offsets, p.weights = lidar2img.data_ptr(), offsets.data_ptr(), weights.data_ptr()
+    p.B, p.N, p.heads, p.head_dim, p.L, p.P = B, N, heads, Dh, L, P
+    p.img_h, p.img_w = img_hw
+    p.x_min, p.x_max, p.y_min, p.y_max, p.z_min, p.z_max = (float(v) for v in bev_range)
+    p.X, p.Y, p.Zref = X, Y, Zref
+    p.out = out.data_ptr()
+    p.hits_out = None if hits is None else hits.data_ptr()
+    if stream is None:
+        stream = torch.cuda.current_stream(value.device).cuda_stream
+    with torch.cuda.device(value.device):
+        flashbev_sca(p, stream)
+    return out
 
 
 def flashbev_workspace_bytes(params: VtParams) -> int:

@@ -892,6 +892,128 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
 }
 
 // ------------------------------------------------------------------------------------------
+// Kernel 3: FlashSCA -- spatial cross-attention with on-the-fly projection (paper Sec. 4.4).  One warp per
+// BEV query: the lanes first project the query's Zref reference heights into all cameras (fp64, the
+// same validity rule as the Sampling-VT operator) and keep the normalised image positions in shared
+// memory; then, for every camera that sees the query, every level and every sampling point, the
+// lanes of a head (head_dim / 4 lanes, 16 bytes of the head's channels each) fetch the four bilinear
+// taps of the value map and accumulate attention weight x bilinear weight x value in fp32.  No
+// per-camera, BEV-shaped tensor (reference points, masks, sampling locations) ever exists in memory.
+
+constexpr int kScaMaxLevels = 8;
+
+struct ScaParams {
+    const float4 *value;   // [B][N][T][D / 4]
+    const float *l2i;
+    const float2 *offsets; // [B][Q][heads][L][P]
+    const float *weights;  // [B][Q][heads][L][P]
+    float4 *out;           // [B][Q][D / 4]
+    int32_t *hits_out;
+    int B, N, heads, Dh, L, P, X, Y, Zref, Himg, Wimg;
+    int lph, hp;           // lanes per head, heads per pass
+    long long T;           // texels per camera (all levels)
+    double x_min, dx, y_min, dy, z_min, dz;
+    int Hl[kScaMaxLevels], Wl[kScaMaxLevels], lvl0[kScaMaxLevels];
+};
+
+template <int V>
+__global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int Q = p.X * p.Y;
+    const long long gq = (long long)blockIdx.x * 4 + warp;  // query index over the batch
+    if (gq >= (long long)p.B * Q) return;
+    const int b = (int)(gq / Q), q = (int)(gq - (long long)b * Q);
+    const int ix = q / p.Y, iy = q - ix * p.Y;
+    const int nref = p.N * p.Zref;
+    const size_t per_warp = (size_t)nref * sizeof(double2) + (((size_t)p.N * sizeof(uint32_t) + 15) & ~(size_t)15);
+    double2 *ref = reinterpret_cast<double2 *>(smem_raw + warp * per_warp);
+    uint32_t *vm = reinterpret_cast<uint32_t *>(smem_raw + warp * per_warp + (size_t)nref * sizeof(double2));
+
+    // ---- reference points: (camera, height) pairs over the lanes
+    for (int n = lane; n < p.N; n += 32) vm[n] = 0u;
+    __syncwarp();
+    const double xw = p.x_min + ((double)ix + 0.5) * p.dx, yw = p.y_min + ((double)iy + 0.5) * p.dy;
+    for (int pr = lane; pr < nref; pr += 32) {
+        const int n = pr / p.Zref, k = pr - n * p.Zref;
+        const float *M = p.l2i + ((size_t)b * p.N + n) * 16;
+        const double zw = p.z_min + ((double)k + 0.5) * p.dz;
+        const double p0 = fma((double)__ldg(M + 2), zw, fma((double)__ldg(M + 1), yw, fma((double)__ldg(M), xw, (double)__ldg(M + 3))));
+        const double p1 = fma((double)__ldg(M + 6), zw, fma((double)__ldg(M + 5), yw, fma((double)__ldg(M + 4), xw, (double)__ldg(M + 7))));
+        const double d = fma((double)__ldg(M + 10), zw, fma((double)__ldg(M + 9), yw, fma((double)__ldg(M + 8), xw, (double)__ldg(M + 11))));
+        const double r = fast_rcp(d);  // d <= 0 or NaN: every test below fails
+        const double u = p0 * r, v = p1 * r;
+        const bool ok = (d > kDepthMin) & (u > 0.0) & (u < (double)p.Wimg) & (v > 0.0) & (v < (double)p.Himg);
+        ref[pr] = make_double2(u / (double)p.Wimg, v / (double)p.Himg);
+        if (ok) atomicOr(&vm[n], 1u << k);
+    }
+    __syncwarp();
+    int hits = 0;
+    for (int n0 = 0; n0 < p.N; n0 += 32)
+        hits += __popc(__ballot_sync(FULL, n0 + lane < p.N && vm[min(n0 + lane, p.N - 1)] != 0u));
+
+    // ---- lanes -> (head, 16-byte slice of the head's channels)
+    const int hsub = lane / p.lph, e4 = lane - hsub * p.lph;
+    const bool lane_role = hsub < p.hp;
+    float4 acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int D4 = p.heads * p.lph;  // float4 per texel
+    const size_t qbase = ((size_t)b * Q + q) * p.heads;
+
+    for (int n = 0; n < p.N; ++n) {
+        const uint32_t mask = vm[n];
+        if (mask == 0u) continue;  // warp-uniform: the camera does not see this query
+        const float4 *vcam = p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4;
+        for (int l = 0; l < p.L; ++l) {
+            const int Hl = p.Hl[l], Wl = p.Wl[l];
+            const float4 *vlev = vcam + (size_t)p.lvl0[l] * D4;
+            for (int pt = 0; pt < p.P; ++pt) {
+                const int k = pt % p.Zref;
+                if (!((mask >> k) & 1u)) continue;  // warp-uniform: this reference height is not visible
+                const double2 rf = ref[n * p.Zref + k];
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const int h = v * p.hp + hsub;
+                    if (!lane_role || h >= p.heads) continue;
+                    const size_t sidx = ((qbase + h) * p.L + l) * p.P + pt;
+                    const float a = __ldg(p.weights + sidx);
+                    const float2 of = __ldg(p.offsets + sidx);
+                    const double px = fma(rf.x, (double)Wl, (double)of.x - 0.5);
+                    const double py = fma(rf.y, (double)Hl, (double)of.y - 0.5);
+                    const double flx = floor(px), fly = floor(py);
+                    // far-away positions: keep the integer conversion defined, every tap is out of range anyway
+                    const int x0 = (int)fmin(fmax(flx, -2.0), (double)Wl), y0 = (int)fmin(fmax(fly, -2.0), (double)Hl);
+                    const float tx = (float)(px - flx), ty = (float)(py - fly);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int xi = x0 + (t & 1), yi = y0 + (t >> 1);
+                        if (xi < 0 || xi > Wl - 1 || yi < 0 || yi > Hl - 1) continue;  // zero padding
+                        const float w = a * ((t & 1) ? tx : 1.f - tx) * ((t >> 1) ? ty : 1.f - ty);
+                        const float4 s = __ldg(vlev + ((size_t)yi * Wl + xi) * D4 + h * p.lph + e4);
+                        acc[v].x = fmaf(w, s.x, acc[v].x);
+                        acc[v].y = fmaf(w, s.y, acc[v].y);
+                        acc[v].z = fmaf(w, s.z, acc[v].z);
+                        acc[v].w = fmaf(w, s.w, acc[v].w);
+                    }
+                }
+            }
+        }
+    }
+    const float g = 1.f / (float)(hits > 1 ? hits : 1);
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int h = v * p.hp + hsub;
+        if (!lane_role || h >= p.heads) continue;
+        __stcs(p.out + ((size_t)b * Q + q) * D4 + h * p.lph + e4,
+               make_float4(acc[v].x * g, acc[v].y * g, acc[v].z * g, acc[v].w * g));
+    }
+    if (p.hits_out && lane == 0) p.hits_out[gq] = hits;
+}
+
+// ------------------------------------------------------------------------------------------
 // host side
 
 thread_local int t_last_launches = 0;
@@ -1284,6 +1406,71 @@ flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params 
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
     t_last_launches = 1;
     t_last_kernel = V == 1 ? "tiled_bwd_v1" : (V == 2 ? "tiled_bwd_v2" : "tiled_bwd_v4");
+    return FLASHBEV_OK;
+}
+
+// ---- FlashSCA ---------------------------------------------------------------------------------
+flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
+{
+    if (!q || q->struct_size < sizeof(flashbev_sca_params)) return FLASHBEV_INVALID_ARG;
+    if (!q->value || !q->level_hw || !q->lidar2img || !q->offsets || !q->weights || !q->out) return FLASHBEV_INVALID_ARG;
+    if (q->B <= 0 || q->N <= 0 || q->heads <= 0 || q->head_dim <= 0 || q->L <= 0 || q->P <= 0) return FLASHBEV_INVALID_ARG;
+    if (q->img_h <= 0 || q->img_w <= 0 || q->X <= 0 || q->Y <= 0 || q->Zref <= 0) return FLASHBEV_INVALID_ARG;
+    if (!(q->x_max > q->x_min) || !(q->y_max > q->y_min) || !(q->z_max > q->z_min)) return FLASHBEV_INVALID_ARG;
+    if (!(q->x_max - q->x_min < 1e300) || !(q->y_max - q->y_min < 1e300) || !(q->z_max - q->z_min < 1e300))
+        return FLASHBEV_INVALID_ARG;
+    if (q->value_dtype != FLASHBEV_F32 && q->value_dtype != FLASHBEV_BF16) return FLASHBEV_INVALID_ARG;
+    ScaParams k = {};
+    long long T = 0;
+    for (int l = 0; l < q->L && l < kScaMaxLevels; ++l) {
+        const int Hl = q->level_hw[2 * l], Wl = q->level_hw[2 * l + 1];
+        if (Hl <= 0 || Wl <= 0) return FLASHBEV_INVALID_ARG;
+        k.Hl[l] = Hl, k.Wl[l] = Wl, k.lvl0[l] = (int)T;
+        T += (long long)Hl * Wl;
+    }
+    if (q->value_dtype != FLASHBEV_F32 || q->L > kScaMaxLevels || q->N > kMaxCams || q->Zref > 32) return FLASHBEV_UNSUPPORTED;
+    if (q->head_dim % 4 || q->head_dim > 128 || (long long)q->N * q->Zref > 1024) return FLASHBEV_UNSUPPORTED;
+    if (T >= 2147483647LL || (double)q->B * q->X * q->Y >= 2147483648.0) return FLASHBEV_UNSUPPORTED;
+    if (((uintptr_t)q->value % 16) || ((uintptr_t)q->out % 16) || ((uintptr_t)q->offsets % 8) ||
+        ((uintptr_t)q->weights % 4) || ((uintptr_t)q->lidar2img % 4) || (q->hits_out && ((uintptr_t)q->hits_out % 4)))
+        return FLASHBEV_MISALIGNED;
+    k.lph = q->head_dim / 4;
+    k.hp = 32 / k.lph;
+    const int V = (q->heads + k.hp - 1) / k.hp;
+    if (V > 4) return FLASHBEV_UNSUPPORTED;
+    k.value = static_cast<const float4 *>(q->value);
+    k.l2i = q->lidar2img;
+    k.offsets = reinterpret_cast<const float2 *>(q->offsets);
+    k.weights = q->weights;
+    k.out = reinterpret_cast<float4 *>(q->out);
+    k.hits_out = q->hits_out;
+    k.B = q->B, k.N = q->N, k.heads = q->heads, k.Dh = q->head_dim, k.L = q->L, k.P = q->P;
+    k.X = q->X, k.Y = q->Y, k.Zref = q->Zref, k.Himg = q->img_h, k.Wimg = q->img_w, k.T = T;
+    k.x_min = q->x_min, k.dx = (q->x_max - q->x_min) / (double)q->X;
+    k.y_min = q->y_min, k.dy = (q->y_max - q->y_min) / (double)q->Y;
+    k.z_min = q->z_min, k.dz = (q->z_max - q->z_min) / (double)q->Zref;
+    const long long queries = (long long)q->B * q->X * q->Y;
+    const long long blocks = (queries + 3) / 4;
+    if (blocks > 2147483647LL) return FLASHBEV_UNSUPPORTED;
+    const size_t per_warp = (size_t)q->N * q->Zref * sizeof(double2) + (((size_t)q->N * sizeof(uint32_t) + 15) & ~(size_t)15);
+    const size_t smem = 4 * per_warp;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    auto launch = [&](auto kern) -> cudaError_t {
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        kern<<<dim3((unsigned)blocks), dim3(128), smem, stream>>>(k);
+        return cudaSuccess;
+    };
+    cudaError_t e;
+    if (V == 1) e = launch(sca_kernel<1>);
+    else if (V == 2) e = launch(sca_kernel<2>);
+    else if (V == 3) e = launch(sca_kernel<3>);
+    else e = launch(sca_kernel<4>);
+    if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+    t_last_launches = 1;
+    t_last_kernel = "sca_f32";
     return FLASHBEV_OK;
 }
 

@@ -206,3 +206,23 @@ def make_inputs(w: Workload, stream: int = 0) -> Inputs:
     if w.dtype == "bf16":
         feats, bits = round_to_bf16(feats)
     return Inputs(w, feats, bits, mats)
+
+
+def make_sca_inputs(P=8, X=200, Y=200, seed=0):
+    """Synthetic inputs of the spatial-cross-attention operator at BEVFormer-base sizes (paper Sec. 4.4:
+    N = 6, C = 256, 8 heads, 200 x 200 queries, Zref = 4, L = 4): six-camera ring rig for 928 x 1600 images,
+    value maps of strides 8-64, standard-normal values and offsets (2 texels sigma), softmax attention weights."""
+    rng = np.random.default_rng(list(SEED_ROOT) + [77, int(seed)])
+    img_hw = (928, 1600)
+    levels = ((116, 200), (58, 100), (29, 50), (15, 25))
+    N, heads, Dh, Zref = 6, 8, 32, 4
+    mats = ring_rig(N, 70.0, img_hw, np.deg2rad(rng.uniform(-2, 2, (1, N))))
+    T = sum(h * w for h, w in levels)
+    value = rng.standard_normal((1, N, T, heads, Dh), dtype=np.float32)
+    Q = X * Y
+    offsets = rng.standard_normal((1, Q, heads, len(levels), P, 2), dtype=np.float32) * np.float32(2.0)
+    logits = rng.standard_normal((1, Q, heads, len(levels) * P), dtype=np.float32)
+    e = np.exp(logits - logits.max(-1, keepdims=True))
+    weights = (e / e.sum(-1, keepdims=True)).reshape(1, Q, heads, len(levels), P).astype(np.float32)
+    return dict(value=value, level_hw=np.array(levels, np.int32), lidar2img=mats, offsets=offsets, weights=weights,
+                img_hw=img_hw, bev_range=(-51.2, 51.2, -51.2, 51.2, -5.0, 3.0), grid=(X, Y, Zref))

@@ -42,7 +42,8 @@ def test_binding_exposes_the_same_names():
 
 
 @pytest.mark.parametrize("cname,mirror", [("flashbev_vt_params", "VtParams"),
-                                          ("flashbev_vt_backward_params", "VtBackwardParams")])
+                                          ("flashbev_vt_backward_params", "VtBackwardParams"),
+                                          ("flashbev_sca_params", "ScaParams")])
 def test_ctypes_struct_matches_the_c_struct(tmp_path, cname, mirror):
     prog = tmp_path / "layout.c"
     cls = getattr(fb, mirror)

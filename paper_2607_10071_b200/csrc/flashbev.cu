@@ -893,14 +893,20 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
 
 // ------------------------------------------------------------------------------------------
 // Kernel 3: FlashSCA -- spatial cross-attention with on-the-fly projection (paper Sec. 4.4).  One warp per
-// BEV query: the lanes first project the query's Zref reference heights into all cameras (fp64, the
-// same validity rule as the Sampling-VT operator) and keep the normalised image positions in shared
-// memory; then, for every camera that sees the query, every level and every sampling point, the
-// lanes of a head (head_dim / 4 lanes, 16 bytes of the head's channels each) fetch the four bilinear
-// taps of the value map and accumulate attention weight x bilinear weight x value in fp32.  No
-// per-camera, BEV-shaped tensor (reference points, masks, sampling locations) ever exists in memory.
+// BEV query, three phases, all warp-local:
+//   1. the lanes project the query's Zref reference heights into all cameras (fp64, the validity rule of
+//      the Sampling-VT operator) and keep the normalised image positions and a per-camera visibility mask
+//      in shared memory;
+//   2. for every camera that sees the query, the lanes turn (head, level, point) triples -- read with
+//      coalesced streaming loads in the order the offsets and weights are stored -- into tap records
+//      {4 value indices, 4 weights} in shared memory: attention weight x bilinear weight, out-of-map taps
+//      clamped to an in-map address with weight 0 (zero padding without predicates);
+//   3. the lanes of a head (head_dim / 4 lanes, 16 bytes of the head's channels each) walk the head's
+//      records: four 128-bit loads and packed fp32 FMAs per record.
+// No per-camera, BEV-shaped tensor (reference points, masks, sampling locations) ever exists in memory.
 
 constexpr int kScaMaxLevels = 8;
+constexpr int kScaMaxChunkPoints = 32;  // sampling points per chunk (bit mask of visible points)
 
 struct ScaParams {
     const float4 *value;   // [B][N][T][D / 4]
@@ -911,10 +917,20 @@ struct ScaParams {
     int32_t *hits_out;
     int B, N, heads, Dh, L, P, X, Y, Zref, Himg, Wimg;
     int lph, hp;           // lanes per head, heads per pass
+    int Pc, pitch;         // points per chunk; records per head in shared memory (L * Pc + 1)
     long long T;           // texels per camera (all levels)
     double x_min, dx, y_min, dy, z_min, dz;
     int Hl[kScaMaxLevels], Wl[kScaMaxLevels], lvl0[kScaMaxLevels];
 };
+
+__host__ __device__ inline size_t sca_warp_smem(int N, int Zref, int heads, int pitch)
+{
+    return (size_t)N * Zref * sizeof(double2) + (((size_t)N * sizeof(uint32_t) + 15) & ~(size_t)15) +
+           (size_t)heads * pitch * 32;
+}
+
+// i / n for 0 <= i < 2^20, given inv = 1 / n in fp32
+__device__ __forceinline__ int small_div(int i, float inv) { return (int)(((float)i + 0.5f) * inv); }
 
 template <int V>
 __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
@@ -928,11 +944,14 @@ __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
     const int b = (int)(gq / Q), q = (int)(gq - (long long)b * Q);
     const int ix = q / p.Y, iy = q - ix * p.Y;
     const int nref = p.N * p.Zref;
-    const size_t per_warp = (size_t)nref * sizeof(double2) + (((size_t)p.N * sizeof(uint32_t) + 15) & ~(size_t)15);
-    double2 *ref = reinterpret_cast<double2 *>(smem_raw + warp * per_warp);
-    uint32_t *vm = reinterpret_cast<uint32_t *>(smem_raw + warp * per_warp + (size_t)nref * sizeof(double2));
+    const int cap = p.heads * p.pitch;
+    unsigned char *mine = smem_raw + warp * sca_warp_smem(p.N, p.Zref, p.heads, p.pitch);
+    double2 *ref = reinterpret_cast<double2 *>(mine);
+    uint32_t *vm = reinterpret_cast<uint32_t *>(mine + (size_t)nref * sizeof(double2));
+    uint4 *rec_i = reinterpret_cast<uint4 *>(mine + (size_t)nref * sizeof(double2) + (((size_t)p.N * 4 + 15) & ~(size_t)15));
+    float4 *rec_w = reinterpret_cast<float4 *>(rec_i + cap);
 
-    // ---- reference points: (camera, height) pairs over the lanes
+    // ---- phase 1: reference points, (camera, height) pairs over the lanes
     for (int n = lane; n < p.N; n += 32) vm[n] = 0u;
     __syncwarp();
     const double xw = p.x_min + ((double)ix + 0.5) * p.dx, yw = p.y_min + ((double)iy + 0.5) * p.dy;
@@ -956,47 +975,103 @@ __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
 
     // ---- lanes -> (head, 16-byte slice of the head's channels)
     const int hsub = lane / p.lph, e4 = lane - hsub * p.lph;
-    const bool lane_role = hsub < p.hp;
-    float4 acc[V];
+    float2 acc[V][2];
+    bool on[V];
+    int hrow[V];  // first record of the lane's head
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v = 0; v < V; ++v) {
+        acc[v][0] = acc[v][1] = make_float2(0.f, 0.f);
+        const int h = v * p.hp + hsub;
+        on[v] = hsub < p.hp && h < p.heads;
+        hrow[v] = (on[v] ? h : 0) * p.pitch;
+    }
     const int D4 = p.heads * p.lph;  // float4 per texel
     const size_t qbase = ((size_t)b * Q + q) * p.heads;
+    const float inv_zref = 1.f / (float)p.Zref;
 
     for (int n = 0; n < p.N; ++n) {
         const uint32_t mask = vm[n];
         if (mask == 0u) continue;  // warp-uniform: the camera does not see this query
-        const float4 *vcam = p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4;
-        for (int l = 0; l < p.L; ++l) {
-            const int Hl = p.Hl[l], Wl = p.Wl[l];
-            const float4 *vlev = vcam + (size_t)p.lvl0[l] * D4;
-            for (int pt = 0; pt < p.P; ++pt) {
-                const int k = pt % p.Zref;
-                if (!((mask >> k) & 1u)) continue;  // warp-uniform: this reference height is not visible
+        const uint4 *vcam = reinterpret_cast<const uint4 *>(p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4) + e4;
+        for (int pt0 = 0; pt0 < p.P; pt0 += p.Pc) {
+            const int npc = min(p.Pc, p.P - pt0);
+            // visible points of the chunk: the reference height a point belongs to must be seen
+            uint32_t vis = 0u;
+            for (int j = 0; j < npc; ++j) {
+                const int pt = pt0 + j;
+                vis |= ((mask >> (pt - small_div(pt, inv_zref) * p.Zref)) & 1u) << j;
+            }
+            if (vis == 0u) continue;
+            __syncwarp();  // the previous chunk's records have been consumed
+            // ---- phase 2: tap records, one (head, level, point) per lane and step
+            const float inv_npc = 1.f / (float)npc, inv_L = 1.f / (float)p.L;
+            const int items = p.heads * p.L * npc;
+            for (int i = lane; i < items; i += 32) {
+                const int hl = small_div(i, inv_npc), j = i - hl * npc;
+                if (!((vis >> j) & 1u)) continue;
+                const int h = small_div(hl, inv_L), l = hl - h * p.L;
+                const int pt = pt0 + j;
+                const int k = pt - small_div(pt, inv_zref) * p.Zref;
+                const size_t sidx = ((qbase + h) * p.L + l) * p.P + pt;
+                const float a = __ldcs(p.weights + sidx);
+                const float2 of = __ldcs(p.offsets + sidx);
                 const double2 rf = ref[n * p.Zref + k];
+                const int Hl = p.Hl[l], Wl = p.Wl[l];
+                const double px = fma(rf.x, (double)Wl, (double)of.x - 0.5);
+                const double py = fma(rf.y, (double)Hl, (double)of.y - 0.5);
+                const double flx = floor(px), fly = floor(py);
+                // far-away positions: keep the integer conversion defined, every tap is out of range anyway
+                const int x0 = (int)fmin(fmax(flx, -2.0), (double)Wl), y0 = (int)fmin(fmax(fly, -2.0), (double)Hl);
+                const float tx = (float)(px - flx), ty = (float)(py - fly);
+                const bool inx0 = x0 >= 0 && x0 <= Wl - 1, inx1 = x0 + 1 >= 0 && x0 + 1 <= Wl - 1;
+                const bool iny0 = y0 >= 0 && y0 <= Hl - 1, iny1 = y0 + 1 >= 0 && y0 + 1 <= Hl - 1;
+                const int xa = min(max(x0, 0), Wl - 1), xb = min(max(x0 + 1, 0), Wl - 1);
+                const int ya = min(max(y0, 0), Hl - 1), yb = min(max(y0 + 1, 0), Hl - 1);
+                const float wx0 = a * (1.f - tx), wx1 = a * tx;
+                float4 w;
+                w.x = inx0 && iny0 ? wx0 * (1.f - ty) : 0.f;
+                w.y = inx1 && iny0 ? wx1 * (1.f - ty) : 0.f;
+                w.z = inx0 && iny1 ? wx0 * ty : 0.f;
+                w.w = inx1 && iny1 ? wx1 * ty : 0.f;
+                const uint32_t hoff = (uint32_t)(h * p.lph);
+                const uint32_t ra = (uint32_t)(p.lvl0[l] + ya * Wl), rb = (uint32_t)(p.lvl0[l] + yb * Wl);
+                uint4 t;
+                t.x = (ra + xa) * D4 + hoff;
+                t.y = (ra + xb) * D4 + hoff;
+                t.z = (rb + xa) * D4 + hoff;
+                t.w = (rb + xb) * D4 + hoff;
+                const int slot = h * p.pitch + l * p.Pc + j;
+                rec_i[slot] = t;
+                rec_w[slot] = w;
+            }
+            __syncwarp();
+            // ---- phase 3: gather, every lane over the records of its heads
+            for (int l = 0; l < p.L; ++l) {
+                for (uint32_t m = vis; m; m &= m - 1u) {
+                    const int slot = l * p.Pc + __ffs(m) - 1;
+                    uint4 ti[V];
+                    float4 tw[V];
+                    uint4 s[V][4];
 #pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    const int h = v * p.hp + hsub;
-                    if (!lane_role || h >= p.heads) continue;
-                    const size_t sidx = ((qbase + h) * p.L + l) * p.P + pt;
-                    const float a = __ldg(p.weights + sidx);
-                    const float2 of = __ldg(p.offsets + sidx);
-                    const double px = fma(rf.x, (double)Wl, (double)of.x - 0.5);
-                    const double py = fma(rf.y, (double)Hl, (double)of.y - 0.5);
-                    const double flx = floor(px), fly = floor(py);
-                    // far-away positions: keep the integer conversion defined, every tap is out of range anyway
-                    const int x0 = (int)fmin(fmax(flx, -2.0), (double)Wl), y0 = (int)fmin(fmax(fly, -2.0), (double)Hl);
-                    const float tx = (float)(px - flx), ty = (float)(py - fly);
+                    for (int v = 0; v < V; ++v) {
+                        ti[v] = rec_i[hrow[v] + slot];
+                        tw[v] = rec_w[hrow[v] + slot];
+                    }
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const int xi = x0 + (t & 1), yi = y0 + (t >> 1);
-                        if (xi < 0 || xi > Wl - 1 || yi < 0 || yi > Hl - 1) continue;  // zero padding
-                        const float w = a * ((t & 1) ? tx : 1.f - tx) * ((t >> 1) ? ty : 1.f - ty);
-                        const float4 s = __ldg(vlev + ((size_t)yi * Wl + xi) * D4 + h * p.lph + e4);
-                        acc[v].x = fmaf(w, s.x, acc[v].x);
-                        acc[v].y = fmaf(w, s.y, acc[v].y);
-                        acc[v].z = fmaf(w, s.z, acc[v].z);
-                        acc[v].w = fmaf(w, s.w, acc[v].w);
+                    for (int v = 0; v < V; ++v) {
+                        if (!on[v]) continue;
+                        s[v][0] = __ldg(vcam + ti[v].x);
+                        s[v][1] = __ldg(vcam + ti[v].y);
+                        s[v][2] = __ldg(vcam + ti[v].z);
+                        s[v][3] = __ldg(vcam + ti[v].w);
+                    }
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        if (!on[v]) continue;
+                        fma_vec<false>(acc[v], s[v][0], make_float2(tw[v].x, tw[v].x));
+                        fma_vec<false>(acc[v], s[v][1], make_float2(tw[v].y, tw[v].y));
+                        fma_vec<false>(acc[v], s[v][2], make_float2(tw[v].z, tw[v].z));
+                        fma_vec<false>(acc[v], s[v][3], make_float2(tw[v].w, tw[v].w));
                     }
                 }
             }
@@ -1005,10 +1080,9 @@ __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
     const float g = 1.f / (float)(hits > 1 ? hits : 1);
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-        const int h = v * p.hp + hsub;
-        if (!lane_role || h >= p.heads) continue;
-        __stcs(p.out + ((size_t)b * Q + q) * D4 + h * p.lph + e4,
-               make_float4(acc[v].x * g, acc[v].y * g, acc[v].z * g, acc[v].w * g));
+        if (!on[v]) continue;
+        __stcs(p.out + ((size_t)b * Q + q) * D4 + (v * p.hp + hsub) * p.lph + e4,
+               make_float4(acc[v][0].x * g, acc[v][0].y * g, acc[v][1].x * g, acc[v][1].y * g));
     }
     if (p.hits_out && lane == 0) p.hits_out[gq] = hits;
 }
@@ -1452,8 +1526,11 @@ flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
     const long long queries = (long long)q->B * q->X * q->Y;
     const long long blocks = (queries + 3) / 4;
     if (blocks > 2147483647LL) return FLASHBEV_UNSUPPORTED;
-    const size_t per_warp = (size_t)q->N * q->Zref * sizeof(double2) + (((size_t)q->N * sizeof(uint32_t) + 15) & ~(size_t)15);
-    const size_t smem = 4 * per_warp;
+    if ((double)T * q->heads * k.lph >= 2147483648.0) return FLASHBEV_UNSUPPORTED;  // 32-bit value indices in the records
+    k.Pc = std::max(1, std::min(std::min(q->P, kScaMaxChunkPoints), 256 / (q->heads * q->L)));
+    k.pitch = q->L * k.Pc + 1;  // odd pitch: the heads of a warp read different shared-memory banks
+    const size_t smem = 4 * sca_warp_smem(q->N, q->Zref, q->heads, k.pitch);
+    if (smem > 200 * 1024) return FLASHBEV_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     auto launch = [&](auto kern) -> cudaError_t {
         if (smem > 48 * 1024) {

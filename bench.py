@@ -288,14 +288,14 @@ def measure_tensorized(torch, w, device, iters=5):
     return {"latency_ms": a.elapsed_time(b) / iters, "peak_mb": (torch.cuda.max_memory_allocated() - base) / 1e6}
 
 
-def measure_sca(torch, device, P, iters=10):
+def measure_sca(torch, device, P, iters=10, chunk_records=0):
     """Latency of the fused spatial cross-attention at BEVFormer-base sizes (inputs ~350 MB+ per call: L2-cold)."""
     from paper_2607_10071_b200 import binding as fb
     c = wl.make_sca_inputs(P=P)
     t = {k: torch.from_numpy(c[k]).to(device) for k in ("value", "lidar2img", "offsets", "weights")}
     out = torch.empty((1, c["grid"][0] * c["grid"][1], 256), dtype=torch.float32, device=device)
     call = lambda: fb.sca(t["value"], c["level_hw"], t["lidar2img"], t["offsets"], t["weights"], c["img_hw"],
-                          c["bev_range"], c["grid"], out=out)
+                          c["bev_range"], c["grid"], out=out, chunk_records=chunk_records)
     for _ in range(3):
         call()
     torch.cuda.synchronize()

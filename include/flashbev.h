@@ -214,7 +214,7 @@ typedef struct flashbev_sca_params {
     const void *value;         /* device, [B][N][T][heads][head_dim], T = sum_l H_l*W_l (levels concatenated,
                                   each level row-major); value_dtype, 16-byte aligned */
     int32_t value_dtype;       /* FLASHBEV_F32 (bf16 values: FLASHBEV_UNSUPPORTED) */
-    int32_t reserved;
+    int32_t chunk_records;     /* tuning: tap records built per pass over a query (shared memory per warp); 0 = default */
     const int32_t *level_hw;   /* HOST, [L][2] = (H_l, W_l); read during the call only; L <= 8 */
     const float *lidar2img;    /* device, [B][N][4][4] float32 */
     const float *offsets;      /* device, [B][X*Y][heads][L][P][2] float32, in texels of level l */

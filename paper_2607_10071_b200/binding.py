@@ -70,7 +70,7 @@ class ScaParams(ctypes.Structure):
     _fields_ = [
         ("struct_size", ctypes.c_size_t),
         ("value", ctypes.c_void_p),
-        ("value_dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("value_dtype", ctypes.c_int32), ("chunk_records", ctypes.c_int32),
         ("level_hw", ctypes.c_void_p),
         ("lidar2img", ctypes.c_void_p),
         ("offsets", ctypes.c_void_p),
@@ -237,7 +237,8 @@ def flashbev_sca(params: ScaParams, stream: int | None = None, check: bool = Tru
     return st
 
 
-def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, out=None, hits=None, stream=None):
+def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, out=None, hits=None, stream=None,
+        chunk_records=0):
     """value: CUDA float32 [B,N,T,heads,Dh]; offsets [B,Q,heads,L,P,2]; weights [B,Q,heads,L,P] (CUDA float32).
     level_hw: sequence of (H_l, W_l).  Returns CUDA float32 [B, Q, heads*Dh] (marshalling only)."""
     import numpy as np
@@ -254,7 +255,7 @@ def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, o
         out = torch.empty((B, X * Y, heads * Dh), dtype=torch.float32, device=value.device)
     p = ScaParams()
     p.struct_size = ctypes.sizeof(ScaParams)
-    p.value, p.value_dtype = value.data_ptr(), F32
+    p.value, p.value_dtype, p.chunk_records = value.data_ptr(), F32, int(chunk_records)
     p.level_hw = lv.ctypes.data
     p.lidar2img, p.offsets, p.weights = lidar2img.data_ptr(), offsets.data_ptr(), weights.data_ptr()
     p.B, p.N, p.heads, p.head_dim, p.L, p.P = B, N, heads, Dh, L, P

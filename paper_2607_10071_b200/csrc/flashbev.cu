@@ -923,17 +923,31 @@ struct ScaParams {
     int Hl[kScaMaxLevels], Wl[kScaMaxLevels], lvl0[kScaMaxLevels];
 };
 
-__host__ __device__ inline size_t sca_warp_smem(int N, int Zref, int heads, int pitch)
+// Shared memory of one warp: reference points, visibility masks, tap records (16 + 16 bytes each) and two
+// staging buffers for the (offset, weight) pairs of a chunk (8 + 4 bytes per head x level x point).
+__host__ __device__ inline size_t sca_warp_smem(int N, int Zref, int heads, int pitch, int items)
 {
     return (size_t)N * Zref * sizeof(double2) + (((size_t)N * sizeof(uint32_t) + 15) & ~(size_t)15) +
-           (size_t)heads * pitch * 32;
+           (size_t)heads * pitch * 32 + 2 * (((size_t)items * 12 + 15) & ~(size_t)15);
 }
+
+__device__ __forceinline__ void cp_async_4(void *dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_8(void *dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // i / n for 0 <= i < 2^20, given inv = 1 / n in fp32
 __device__ __forceinline__ int small_div(int i, float inv) { return (int)(((float)i + 0.5f) * inv); }
 
 template <int V>
-__global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
+__global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr unsigned FULL = 0xffffffffu;
@@ -945,11 +959,33 @@ __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
     const int ix = q / p.Y, iy = q - ix * p.Y;
     const int nref = p.N * p.Zref;
     const int cap = p.heads * p.pitch;
-    unsigned char *mine = smem_raw + warp * sca_warp_smem(p.N, p.Zref, p.heads, p.pitch);
+    const int max_items = p.heads * p.L * p.Pc;
+    const size_t stage_bytes = ((size_t)max_items * 12 + 15) & ~(size_t)15;
+    unsigned char *mine = smem_raw + warp * sca_warp_smem(p.N, p.Zref, p.heads, p.pitch, max_items);
     double2 *ref = reinterpret_cast<double2 *>(mine);
     uint32_t *vm = reinterpret_cast<uint32_t *>(mine + (size_t)nref * sizeof(double2));
     uint4 *rec_i = reinterpret_cast<uint4 *>(mine + (size_t)nref * sizeof(double2) + (((size_t)p.N * 4 + 15) & ~(size_t)15));
     float4 *rec_w = reinterpret_cast<float4 *>(rec_i + cap);
+    unsigned char *stage = reinterpret_cast<unsigned char *>(rec_w + cap);  // [2][offsets: items x 8 | weights: items x 4]
+
+    const size_t qbase = ((size_t)b * Q + q) * p.heads;
+    const float inv_L = 1.f / (float)p.L, inv_zref = 1.f / (float)p.Zref;
+    // asynchronous copy of one chunk's offsets and weights, item i = (head * L + level) * npc + point
+    const auto stage_chunk = [&](int pt0, int buf) {
+        const int npc = min(p.Pc, p.P - pt0);
+        const float inv_npc = 1.f / (float)npc;
+        const int items = p.heads * p.L * npc;
+        float2 *so = reinterpret_cast<float2 *>(stage + buf * stage_bytes);
+        float *sw = reinterpret_cast<float *>(so + max_items);
+        for (int i = lane; i < items; i += 32) {
+            const int hl = small_div(i, inv_npc), j = i - hl * npc;
+            const size_t sidx = (qbase * p.L + hl) * p.P + pt0 + j;
+            cp_async_8(so + i, p.offsets + sidx);
+            cp_async_4(sw + i, p.weights + sidx);
+        }
+        cp_async_commit();
+    };
+    stage_chunk(0, 0);
 
     // ---- phase 1: reference points, (camera, height) pairs over the lanes
     for (int n = lane; n < p.N; n += 32) vm[n] = 0u;
@@ -986,15 +1022,24 @@ __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
         hrow[v] = (on[v] ? h : 0) * p.pitch;
     }
     const int D4 = p.heads * p.lph;  // float4 per texel
-    const size_t qbase = ((size_t)b * Q + q) * p.heads;
-    const float inv_zref = 1.f / (float)p.Zref;
 
-    for (int n = 0; n < p.N; ++n) {
-        const uint32_t mask = vm[n];
-        if (mask == 0u) continue;  // warp-uniform: the camera does not see this query
-        const uint4 *vcam = reinterpret_cast<const uint4 *>(p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4) + e4;
-        for (int pt0 = 0; pt0 < p.P; pt0 += p.Pc) {
-            const int npc = min(p.Pc, p.P - pt0);
+    for (int pt0 = 0, c = 0; pt0 < p.P; pt0 += p.Pc, ++c) {
+        const int npc = min(p.Pc, p.P - pt0);
+        // the next chunk's offsets and weights travel while this one is worked on
+        if (pt0 + p.Pc < p.P) {
+            stage_chunk(pt0 + p.Pc, (c + 1) & 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncwarp();
+        const float2 *so = reinterpret_cast<const float2 *>(stage + (c & 1) * stage_bytes);
+        const float *sw = reinterpret_cast<const float *>(so + max_items);
+        const float inv_npc = 1.f / (float)npc;
+        const int items = p.heads * p.L * npc;
+        for (int n = 0; n < p.N; ++n) {
+            const uint32_t mask = vm[n];
+            if (mask == 0u) continue;  // warp-uniform: the camera does not see this query
             // visible points of the chunk: the reference height a point belongs to must be seen
             uint32_t vis = 0u;
             for (int j = 0; j < npc; ++j) {
@@ -1002,19 +1047,17 @@ __global__ void __launch_bounds__(128) sca_kernel(const ScaParams p)
                 vis |= ((mask >> (pt - small_div(pt, inv_zref) * p.Zref)) & 1u) << j;
             }
             if (vis == 0u) continue;
-            __syncwarp();  // the previous chunk's records have been consumed
+            const uint4 *vcam = reinterpret_cast<const uint4 *>(p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4) + e4;
+            __syncwarp();  // the previous records have been consumed
             // ---- phase 2: tap records, one (head, level, point) per lane and step
-            const float inv_npc = 1.f / (float)npc, inv_L = 1.f / (float)p.L;
-            const int items = p.heads * p.L * npc;
             for (int i = lane; i < items; i += 32) {
                 const int hl = small_div(i, inv_npc), j = i - hl * npc;
                 if (!((vis >> j) & 1u)) continue;
                 const int h = small_div(hl, inv_L), l = hl - h * p.L;
                 const int pt = pt0 + j;
                 const int k = pt - small_div(pt, inv_zref) * p.Zref;
-                const size_t sidx = ((qbase + h) * p.L + l) * p.P + pt;
-                const float a = __ldcs(p.weights + sidx);
-                const float2 of = __ldcs(p.offsets + sidx);
+                const float a = sw[i];
+                const float2 of = so[i];
                 const double2 rf = ref[n * p.Zref + k];
                 const int Hl = p.Hl[l], Wl = p.Wl[l];
                 const double px = fma(rf.x, (double)Wl, (double)of.x - 0.5);
@@ -1527,9 +1570,11 @@ flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
     const long long blocks = (queries + 3) / 4;
     if (blocks > 2147483647LL) return FLASHBEV_UNSUPPORTED;
     if ((double)T * q->heads * k.lph >= 2147483648.0) return FLASHBEV_UNSUPPORTED;  // 32-bit value indices in the records
-    k.Pc = std::max(1, std::min(std::min(q->P, kScaMaxChunkPoints), 256 / (q->heads * q->L)));
+    if (q->chunk_records < 0) return FLASHBEV_INVALID_ARG;
+    const int chunk_records = q->chunk_records > 0 ? q->chunk_records : 128;
+    k.Pc = std::max(1, std::min(std::min(q->P, kScaMaxChunkPoints), chunk_records / (q->heads * q->L)));
     k.pitch = q->L * k.Pc + 1;  // odd pitch: the heads of a warp read different shared-memory banks
-    const size_t smem = 4 * sca_warp_smem(q->N, q->Zref, q->heads, k.pitch);
+    const size_t smem = 4 * sca_warp_smem(q->N, q->Zref, q->heads, k.pitch, q->heads * q->L * k.Pc);
     if (smem > 200 * 1024) return FLASHBEV_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     auto launch = [&](auto kern) -> cudaError_t {

@@ -923,12 +923,13 @@ struct ScaParams {
     int Hl[kScaMaxLevels], Wl[kScaMaxLevels], lvl0[kScaMaxLevels];
 };
 
-// Shared memory of one warp: reference points, visibility masks, tap records (16 + 16 bytes each) and two
-// staging buffers for the (offset, weight) pairs of a chunk (8 + 4 bytes per head x level x point).
-__host__ __device__ inline size_t sca_warp_smem(int N, int Zref, int heads, int pitch, int items)
+// Shared memory of one warp: reference points, visibility masks, tap records (16 + 16 bytes each), the
+// texel positions of the references of one camera (16 bytes per height x level) and two staging buffers
+// for the (offset, weight) pairs of a chunk (8 + 4 bytes per head x level x point).
+__host__ __device__ inline size_t sca_warp_smem(int N, int Zref, int heads, int pitch, int items, int L)
 {
     return (size_t)N * Zref * sizeof(double2) + (((size_t)N * sizeof(uint32_t) + 15) & ~(size_t)15) +
-           (size_t)heads * pitch * 32 + 2 * (((size_t)items * 12 + 15) & ~(size_t)15);
+           (size_t)heads * pitch * 32 + (size_t)Zref * L * 16 + 2 * (((size_t)items * 12 + 15) & ~(size_t)15);
 }
 
 __device__ __forceinline__ void cp_async_4(void *dst, const void *src)
@@ -946,40 +947,52 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // i / n for 0 <= i < 2^20, given inv = 1 / n in fp32
 __device__ __forceinline__ int small_div(int i, float inv) { return (int)(((float)i + 0.5f) * inv); }
 
-template <int V>
+// EVEN: every lane has a head in every pass (heads = V * heads per pass, 32 lanes all used)
+template <int V, bool EVEN>
 __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int Q = p.X * p.Y;
-    const long long gq = (long long)blockIdx.x * 4 + warp;  // query index over the batch
-    if (gq >= (long long)p.B * Q) return;
-    const int b = (int)(gq / Q), q = (int)(gq - (long long)b * Q);
-    const int ix = q / p.Y, iy = q - ix * p.Y;
+    const int max_items = p.heads * p.L * p.Pc;
+
+    // ---- per-CTA table: item i = (head * L + level) * Pc + point  ->  head | level | point | point % Zref
+    uint32_t *dec = reinterpret_cast<uint32_t *>(smem_raw);
+    for (int i = threadIdx.x; i < max_items; i += blockDim.x) {
+        const int hl = i / p.Pc, j = i - hl * p.Pc;
+        const int h = hl / p.L, l = hl - h * p.L;
+        dec[i] = ((uint32_t)h << 24) | ((uint32_t)l << 16) | ((uint32_t)(j % p.Zref) << 8) | (uint32_t)j;
+    }
+    __syncthreads();
+
+    const unsigned Q = (unsigned)(p.X * p.Y);
+    const unsigned gq = blockIdx.x * 4u + (unsigned)warp;  // query index over the batch (< 2^31, checked by the host)
+    if (gq >= (unsigned)p.B * Q) return;
+    const unsigned b = gq / Q, q = gq - b * Q;
+    const int ix = (int)(q / (unsigned)p.Y), iy = (int)(q - (unsigned)ix * (unsigned)p.Y);
     const int nref = p.N * p.Zref;
     const int cap = p.heads * p.pitch;
-    const int max_items = p.heads * p.L * p.Pc;
     const size_t stage_bytes = ((size_t)max_items * 12 + 15) & ~(size_t)15;
-    unsigned char *mine = smem_raw + warp * sca_warp_smem(p.N, p.Zref, p.heads, p.pitch, max_items);
+    unsigned char *mine = smem_raw + (((size_t)max_items * 4 + 15) & ~(size_t)15) +
+                          warp * sca_warp_smem(p.N, p.Zref, p.heads, p.pitch, max_items, p.L);
     double2 *ref = reinterpret_cast<double2 *>(mine);
     uint32_t *vm = reinterpret_cast<uint32_t *>(mine + (size_t)nref * sizeof(double2));
     uint4 *rec_i = reinterpret_cast<uint4 *>(mine + (size_t)nref * sizeof(double2) + (((size_t)p.N * 4 + 15) & ~(size_t)15));
     float4 *rec_w = reinterpret_cast<float4 *>(rec_i + cap);
-    unsigned char *stage = reinterpret_cast<unsigned char *>(rec_w + cap);  // [2][offsets: items x 8 | weights: items x 4]
+    int4 *base_tab = reinterpret_cast<int4 *>(rec_w + cap);                       // [Zref][L]: texel position of a reference
+    unsigned char *stage = reinterpret_cast<unsigned char *>(base_tab + p.Zref * p.L);  // [2][offsets | weights]
 
-    const size_t qbase = ((size_t)b * Q + q) * p.heads;
-    const float inv_L = 1.f / (float)p.L, inv_zref = 1.f / (float)p.Zref;
-    // asynchronous copy of one chunk's offsets and weights, item i = (head * L + level) * npc + point
+    const size_t qrow = ((size_t)b * Q + q) * (size_t)(p.heads * p.L);  // first (head, level) row of the query
+    // asynchronous copy of one chunk's offsets and weights into item order
     const auto stage_chunk = [&](int pt0, int buf) {
         const int npc = min(p.Pc, p.P - pt0);
-        const float inv_npc = 1.f / (float)npc;
-        const int items = p.heads * p.L * npc;
         float2 *so = reinterpret_cast<float2 *>(stage + buf * stage_bytes);
         float *sw = reinterpret_cast<float *>(so + max_items);
-        for (int i = lane; i < items; i += 32) {
-            const int hl = small_div(i, inv_npc), j = i - hl * npc;
-            const size_t sidx = (qbase * p.L + hl) * p.P + pt0 + j;
+        for (int i = lane; i < max_items; i += 32) {
+            const uint32_t t = dec[i];
+            const int j = (int)(t & 0xffu);
+            if (j >= npc) continue;
+            const size_t sidx = (qrow + (t >> 24) * p.L + ((t >> 16) & 0xffu)) * p.P + pt0 + j;
             cp_async_8(so + i, p.offsets + sidx);
             cp_async_4(sw + i, p.weights + sidx);
         }
@@ -1018,10 +1031,11 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
     for (int v = 0; v < V; ++v) {
         acc[v][0] = acc[v][1] = make_float2(0.f, 0.f);
         const int h = v * p.hp + hsub;
-        on[v] = hsub < p.hp && h < p.heads;
+        on[v] = EVEN || (hsub < p.hp && h < p.heads);
         hrow[v] = (on[v] ? h : 0) * p.pitch;
     }
     const int D4 = p.heads * p.lph;  // float4 per texel
+    const int nbase = p.Zref * p.L;
 
     for (int pt0 = 0, c = 0; pt0 < p.P; pt0 += p.Pc, ++c) {
         const int npc = min(p.Pc, p.P - pt0);
@@ -1035,39 +1049,46 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
         __syncwarp();
         const float2 *so = reinterpret_cast<const float2 *>(stage + (c & 1) * stage_bytes);
         const float *sw = reinterpret_cast<const float *>(so + max_items);
-        const float inv_npc = 1.f / (float)npc;
-        const int items = p.heads * p.L * npc;
+        const int k0 = pt0 % p.Zref;
+        const int klane = (pt0 + lane) % p.Zref;  // reference height of the chunk's point `lane`
         for (int n = 0; n < p.N; ++n) {
             const uint32_t mask = vm[n];
             if (mask == 0u) continue;  // warp-uniform: the camera does not see this query
             // visible points of the chunk: the reference height a point belongs to must be seen
-            uint32_t vis = 0u;
-            for (int j = 0; j < npc; ++j) {
-                const int pt = pt0 + j;
-                vis |= ((mask >> (pt - small_div(pt, inv_zref) * p.Zref)) & 1u) << j;
-            }
+            const uint32_t vis = __ballot_sync(FULL, lane < npc && ((mask >> klane) & 1u));
             if (vis == 0u) continue;
             const uint4 *vcam = reinterpret_cast<const uint4 *>(p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4) + e4;
-            __syncwarp();  // the previous records have been consumed
+            __syncwarp();  // the previous records and reference positions have been consumed
+            // texel position of every visible reference on every level: integer part and fraction
+            for (int e = lane; e < nbase; e += 32) {
+                const int k = e / p.L, l = e - k * p.L;
+                if (!((mask >> k) & 1u)) continue;
+                const double2 rf = ref[n * p.Zref + k];  // inside (0, 1)^2
+                const double bx = fma(rf.x, (double)p.Wl[l], -0.5), by = fma(rf.y, (double)p.Hl[l], -0.5);
+                const double fbx = floor(bx), fby = floor(by);
+                base_tab[e] = make_int4((int)fbx, (int)fby, __float_as_int((float)(bx - fbx)), __float_as_int((float)(by - fby)));
+            }
+            __syncwarp();
             // ---- phase 2: tap records, one (head, level, point) per lane and step
-            for (int i = lane; i < items; i += 32) {
-                const int hl = small_div(i, inv_npc), j = i - hl * npc;
-                if (!((vis >> j) & 1u)) continue;
-                const int h = small_div(hl, inv_L), l = hl - h * p.L;
-                const int pt = pt0 + j;
-                const int k = pt - small_div(pt, inv_zref) * p.Zref;
+            for (int i = lane; i < max_items; i += 32) {
+                const uint32_t t = dec[i];
+                const int j = (int)(t & 0xffu);
+                if (j >= npc || !((vis >> j) & 1u)) continue;
+                const int h = (int)(t >> 24), l = (int)((t >> 16) & 0xffu);
+                int k = (int)((t >> 8) & 0xffu) + k0;
+                k = k >= p.Zref ? k - p.Zref : k;
                 const float a = sw[i];
                 const float2 of = so[i];
-                const double2 rf = ref[n * p.Zref + k];
+                const int4 bs = base_tab[k * p.L + l];
                 const int Hl = p.Hl[l], Wl = p.Wl[l];
-                const double px = fma(rf.x, (double)Wl, (double)of.x - 0.5);
-                const double py = fma(rf.y, (double)Hl, (double)of.y - 0.5);
-                const double flx = floor(px), fly = floor(py);
-                // far-away positions: keep the integer conversion defined, every tap is out of range anyway
-                const int x0 = (int)fmin(fmax(flx, -2.0), (double)Wl), y0 = (int)fmin(fmax(fly, -2.0), (double)Hl);
-                const float tx = (float)(px - flx), ty = (float)(py - fly);
-                const bool inx0 = x0 >= 0 && x0 <= Wl - 1, inx1 = x0 + 1 >= 0 && x0 + 1 <= Wl - 1;
-                const bool iny0 = y0 >= 0 && y0 <= Hl - 1, iny1 = y0 + 1 >= 0 && y0 + 1 <= Hl - 1;
+                // position = integer base + (fraction + offset); absurd offsets are clamped, their taps are all outside
+                const float sx = fminf(fmaxf(__int_as_float(bs.z) + of.x, -65536.f), 65536.f);
+                const float sy = fminf(fmaxf(__int_as_float(bs.w) + of.y, -65536.f), 65536.f);
+                const float flx = floorf(sx), fly = floorf(sy);
+                const float tx = sx - flx, ty = sy - fly;
+                const int x0 = bs.x + (int)flx, y0 = bs.y + (int)fly;
+                const bool inx0 = (unsigned)x0 < (unsigned)Wl, inx1 = (unsigned)(x0 + 1) < (unsigned)Wl;
+                const bool iny0 = (unsigned)y0 < (unsigned)Hl, iny1 = (unsigned)(y0 + 1) < (unsigned)Hl;
                 const int xa = min(max(x0, 0), Wl - 1), xb = min(max(x0 + 1, 0), Wl - 1);
                 const int ya = min(max(y0, 0), Hl - 1), yb = min(max(y0 + 1, 0), Hl - 1);
                 const float wx0 = a * (1.f - tx), wx1 = a * tx;
@@ -1078,14 +1099,13 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
                 w.w = inx1 && iny1 ? wx1 * ty : 0.f;
                 const uint32_t hoff = (uint32_t)(h * p.lph);
                 const uint32_t ra = (uint32_t)(p.lvl0[l] + ya * Wl), rb = (uint32_t)(p.lvl0[l] + yb * Wl);
-                uint4 t;
-                t.x = (ra + xa) * D4 + hoff;
-                t.y = (ra + xb) * D4 + hoff;
-                t.z = (rb + xa) * D4 + hoff;
-                t.w = (rb + xb) * D4 + hoff;
-                const int slot = h * p.pitch + l * p.Pc + j;
-                rec_i[slot] = t;
-                rec_w[slot] = w;
+                uint4 ti;
+                ti.x = (ra + xa) * D4 + hoff;
+                ti.y = (ra + xb) * D4 + hoff;
+                ti.z = (rb + xa) * D4 + hoff;
+                ti.w = (rb + xb) * D4 + hoff;
+                rec_i[i + h] = ti;  // = head * pitch + level * Pc + point
+                rec_w[i + h] = w;
             }
             __syncwarp();
             // ---- phase 3: gather, every lane over the records of its heads
@@ -1574,7 +1594,8 @@ flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
     const int chunk_records = q->chunk_records > 0 ? q->chunk_records : 128;
     k.Pc = std::max(1, std::min(std::min(q->P, kScaMaxChunkPoints), chunk_records / (q->heads * q->L)));
     k.pitch = q->L * k.Pc + 1;  // odd pitch: the heads of a warp read different shared-memory banks
-    const size_t smem = 4 * sca_warp_smem(q->N, q->Zref, q->heads, k.pitch, q->heads * q->L * k.Pc);
+    const int items = q->heads * q->L * k.Pc;
+    const size_t smem = (((size_t)items * 4 + 15) & ~(size_t)15) + 4 * sca_warp_smem(q->N, q->Zref, q->heads, k.pitch, items, q->L);
     if (smem > 200 * 1024) return FLASHBEV_UNSUPPORTED;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     auto launch = [&](auto kern) -> cudaError_t {
@@ -1586,10 +1607,11 @@ flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
         return cudaSuccess;
     };
     cudaError_t e;
-    if (V == 1) e = launch(sca_kernel<1>);
-    else if (V == 2) e = launch(sca_kernel<2>);
-    else if (V == 3) e = launch(sca_kernel<3>);
-    else e = launch(sca_kernel<4>);
+    const bool even = k.hp * k.lph == 32 && q->heads == V * k.hp;
+    if (V == 1) e = even ? launch(sca_kernel<1, true>) : launch(sca_kernel<1, false>);
+    else if (V == 2) e = even ? launch(sca_kernel<2, true>) : launch(sca_kernel<2, false>);
+    else if (V == 3) e = even ? launch(sca_kernel<3, true>) : launch(sca_kernel<3, false>);
+    else e = even ? launch(sca_kernel<4, true>) : launch(sca_kernel<4, false>);
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
     t_last_launches = 1;
     t_last_kernel = "sca_f32";

@@ -233,6 +233,38 @@ typedef struct flashbev_sca_params {
 
 flashbev_status flashbev_sca(const flashbev_sca_params *p, void *stream);
 
+/* ---- multi-resolution gathering ------------------------------------------------------------
+ * The paper names gathering from several feature resolutions as future work (Sec. 5) and gives no
+ * formula; the operation built here is the plain sum over the levels of a feature pyramid,
+ *
+ *     out = sum_l  SamplingVT(features_l; feat_h_l x feat_w_l),
+ *
+ * every level sampled at the same voxel centres with the same matrices, validity rule, interpolation
+ * and reduce mode as the single-level operator (for the two mean modes every level is normalised
+ * by itself before the sum).  One launch per level on `stream`; level 0 overwrites `out`, the others
+ * add to it, so nothing is allocated and no workspace is needed.
+ *
+ *   base      all arguments of the single-level call; its `features`, `feat_h`, `feat_w` are ignored.
+ *             `out_dtype` must be FLASHBEV_F32 (partial sums are not rounded); `valid_count_out`, if
+ *             given, receives the counts of level 0.
+ *   levels    number of levels, 1..FLASHBEV_MAX_LEVELS
+ *   features  HOST array of `levels` DEVICE pointers, each a tensor of the layout and dtype of `base`
+ *             with C channels and its own map size; read during the call only
+ *   feat_hw   HOST array [levels][2] = (feat_h_l, feat_w_l); read during the call only
+ * Alignment and size rules are those of flashbev_sampling_vt, checked for every level before the
+ * first launch.  flashbev_last_launch_count() reports `levels` afterwards. */
+#define FLASHBEV_MAX_LEVELS 8
+typedef struct flashbev_vt_multires_params {
+    size_t struct_size;              /* sizeof(flashbev_vt_multires_params) of the caller's header */
+    const flashbev_vt_params *base;  /* HOST */
+    int32_t levels;
+    int32_t reserved;
+    const void *const *features;     /* HOST array of DEVICE pointers */
+    const int32_t *feat_hw;          /* HOST, [levels][2] */
+} flashbev_vt_multires_params;
+
+flashbev_status flashbev_sampling_vt_multires(const flashbev_vt_multires_params *p, void *stream);
+
 /* Number of kernels the last successful call of flashbev_sampling_vt[_host] on this thread
  * enqueued (always 1), and a short name of the kernel instance it chose (static storage). */
 int flashbev_last_launch_count(void);

@@ -152,3 +152,20 @@ def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, t
     if rc != 0:
         raise ValueError(f"flashbev_oracle_sca rejected its arguments (status {rc})")
     return out, hits, flagged
+
+
+def sampling_vt_multires(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM, threads=0) -> OracleResult:
+    """Multi-resolution gathering, defined as the plain sum over the pyramid levels of the single-level
+    operator (every level normalised by itself in the mean modes).  The paper only names the idea as
+    future work; this is the definition the CUDA entry point documents.
+
+    features: sequence of float32 arrays [B, N, Hf_l, Wf_l, C].  count/flagged/interior/nzbins are those of
+    level 0, except `flagged`, which is the per-cell maximum over the levels.
+    """
+    res = [sampling_vt(f, lidar2img, img_hw, bev_range, grid, reduce, threads) for f in features]
+    out = res[0].out.copy()
+    flagged = res[0].flagged.copy()
+    for r in res[1:]:
+        out += r.out
+        flagged = np.maximum(flagged, r.flagged)
+    return OracleResult(out, res[0].count, flagged, res[0].sumw, res[0].interior, res[0].nzbins)

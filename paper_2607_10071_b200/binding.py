@@ -87,6 +87,20 @@ class ScaParams(ctypes.Structure):
     ]
 
 
+class VtMultiresParams(ctypes.Structure):
+    """ctypes mirror of ``flashbev_vt_multires_params``."""
+    _fields_ = [
+        ("struct_size", ctypes.c_size_t),
+        ("base", ctypes.POINTER(VtParams)),
+        ("levels", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("features", ctypes.POINTER(ctypes.c_void_p)),
+        ("feat_hw", ctypes.POINTER(ctypes.c_int32)),
+    ]
+
+
+MAX_LEVELS = 8
+
+
 class FlashBevError(RuntimeError):
     def __init__(self, status: int, what: str):
         super().__init__(f"{what}: {status_string(status)} (status {status})")
@@ -114,6 +128,8 @@ def lib() -> ctypes.CDLL:
         L.flashbev_sampling_vt_host_static.argtypes = [P, ctypes.c_void_p]
         L.flashbev_sampling_vt_backward.restype = ctypes.c_int
         L.flashbev_sampling_vt_backward.argtypes = [ctypes.POINTER(VtBackwardParams), ctypes.c_void_p]
+        L.flashbev_sampling_vt_multires.restype = ctypes.c_int
+        L.flashbev_sampling_vt_multires.argtypes = [ctypes.POINTER(VtMultiresParams), ctypes.c_void_p]
         L.flashbev_sca.restype = ctypes.c_int
         L.flashbev_sca.argtypes = [ctypes.POINTER(ScaParams), ctypes.c_void_p]
         L.flashbev_workspace_bytes.restype = ctypes.c_size_t
@@ -182,6 +198,25 @@ def flashbev_sampling_vt_host_static(params: VtParams, stream: int | None = None
     st = lib().flashbev_sampling_vt_host_static(ctypes.byref(params), ctypes.c_void_p(stream or 0))
     if check and st != OK:
         raise FlashBevError(st, "flashbev_sampling_vt_host_static")
+    return st
+
+
+def flashbev_sampling_vt_multires(base: VtParams, feature_ptrs, feat_hws, stream: int | None = None,
+                                  check: bool = True) -> int:
+    """Sum of the operator over the levels of a feature pyramid: ``feature_ptrs`` are device pointers,
+    ``feat_hws`` the (feat_h, feat_w) of every level; ``base`` carries everything else."""
+    n = len(feature_ptrs)
+    q = VtMultiresParams()
+    q.struct_size = ctypes.sizeof(VtMultiresParams)
+    q.base = ctypes.pointer(base)
+    q.levels = n
+    ptrs = (ctypes.c_void_p * max(n, 1))(*[int(v) for v in feature_ptrs])
+    hw = (ctypes.c_int32 * max(2 * n, 2))(*[int(v) for pair in feat_hws for v in pair])
+    q.features = ctypes.cast(ptrs, ctypes.POINTER(ctypes.c_void_p))
+    q.feat_hw = ctypes.cast(hw, ctypes.POINTER(ctypes.c_int32))
+    st = lib().flashbev_sampling_vt_multires(ctypes.byref(q), ctypes.c_void_p(stream or 0))
+    if check and st != OK:
+        raise FlashBevError(st, "flashbev_sampling_vt_multires")
     return st
 
 
@@ -325,4 +360,41 @@ def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM,
         stream = torch.cuda.current_stream(features.device).cuda_stream
     with torch.cuda.device(features.device):
         flashbev_sampling_vt(p, stream)
+    return out
+
+
+def sampling_vt_multires(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM, out=None,
+                         valid_count=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0), stream=None, layout=NHWC):
+    """features: sequence of CUDA tensors, one per pyramid level, each [B,N,Hf_l,Wf_l,C] (NHWC) or
+    [B,N,C,Hf_l,Wf_l] (NCHW) of one dtype.  Returns the float32 sum over the levels (marshalling only)."""
+    import torch
+
+    f0 = features[0]
+    for f in features:
+        if not f.is_cuda or not f.is_contiguous() or f.dtype != f0.dtype:
+            raise ValueError("every level must be a contiguous CUDA tensor of the same dtype")
+    if f0.dtype == torch.float32:
+        dt = F32
+    elif f0.dtype == torch.bfloat16:
+        dt = BF16
+    else:
+        raise ValueError("features must be float32 or bfloat16")
+    if not lidar2img.is_cuda or lidar2img.dtype != torch.float32 or not lidar2img.is_contiguous():
+        raise ValueError("lidar2img must be a contiguous CUDA float32 tensor")
+    if layout == NHWC:
+        B, N, _, _, C = f0.shape
+        hws = [(f.shape[2], f.shape[3]) for f in features]
+    else:
+        B, N, C, _, _ = f0.shape
+        hws = [(f.shape[3], f.shape[4]) for f in features]
+    X, Y, Z = grid
+    if out is None:
+        out = torch.empty((B, X, Y, C) if layout == NHWC else (B, C, X, Y), dtype=torch.float32, device=f0.device)
+    base = make_params(f0.data_ptr(), dt, lidar2img.data_ptr(), B, N, C, hws[0], img_hw, bev_range, (X, Y, Z),
+                       reduce, out.data_ptr(), None if valid_count is None else valid_count.data_ptr(),
+                       kernel, tune, layout, F32)
+    if stream is None:
+        stream = torch.cuda.current_stream(f0.device).cuda_stream
+    with torch.cuda.device(f0.device):
+        flashbev_sampling_vt_multires(base, [f.data_ptr() for f in features], hws, stream)
     return out

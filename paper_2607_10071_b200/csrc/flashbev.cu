@@ -40,6 +40,7 @@ struct KParams {
     float *gfeat;               // backward: gradient of the features [B][N][Hf][Wf][C], fp32, pre-zeroed
     int B, N, C, Hf, Wf, X, Y, Z, reduce;
     int out_bf16;               // store the output as bfloat16 (round to nearest even) instead of float32
+    int accumulate;             // add the result to the fp32 output instead of overwriting it (multi-resolution levels)
     double sx, sy;              // image px -> feature px
     double x_min, dx, y_min, dy, z_min, dz;
     // tiled kernel only
@@ -206,6 +207,10 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
         }
     } else {
         float *o = p.out + (size_t)cell * p.C + c0;
+        if (p.accumulate) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) acc[i] += o[i];
+        }
         if (VEC == 1) {
             o[0] = acc[0];
         } else {
@@ -264,7 +269,7 @@ __global__ void __launch_bounds__(256) vt_per_output_nchw_kernel(const KParams p
     }
     if (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) acc *= 1.f / (float)(count > 1 ? count : 1);
     if (p.out_bf16) reinterpret_cast<uint16_t *>(p.out)[gid] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
-    else p.out[gid] = acc;
+    else p.out[gid] = p.accumulate ? acc + p.out[gid] : acc;
     if (p.count_out && c == 0) p.count_out[((size_t)b * p.X + ix) * p.Y + iy] = count;
 }
 
@@ -864,6 +869,10 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                                         val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
                                     }
                                     val.x *= g, val.y *= g, val.z *= g, val.w *= g;
+                                    if (p.accumulate) {  // one sub-block per warp: `dst` still holds the other levels' sum
+                                        const float4 prev = *dst;
+                                        val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
+                                    }
                                     if (p.out_bf16) {  // only with one sub-block per warp: this is the single, final store
                                         uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C;
                                         *reinterpret_cast<uint2 *>(ob + (size_t)vi * (PV * 2) + e * 2) =
@@ -1193,9 +1202,10 @@ flashbev_status check_alignment(const flashbev_vt_params *p)
     return FLASHBEV_OK;
 }
 
-KParams base_params(const flashbev_vt_params *p)
+KParams base_params(const flashbev_vt_params *p, bool accumulate = false)
 {
     KParams k = {};
+    k.accumulate = accumulate;
     k.feat = p->features;
     k.l2i = p->lidar2img;
     k.out = static_cast<float *>(p->out);
@@ -1211,9 +1221,9 @@ KParams base_params(const flashbev_vt_params *p)
     return k;
 }
 
-flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stream)
+flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false)
 {
-    const KParams k = base_params(p);
+    const KParams k = base_params(p, accumulate);
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     if (p->layout == FLASHBEV_NCHW) {
         const long long threads = (long long)p->B * p->C * p->X * p->Y;
@@ -1301,9 +1311,10 @@ cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t sm
 }
 
 // Chooses the channel mapping, super-block shape, chunking and grid of the tiled kernel.
-flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V, int &warps, dim3 &grid, size_t &smem)
+flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V, int &warps, dim3 &grid, size_t &smem,
+                                bool accumulate = false)
 {
-    k = base_params(p);
+    k = base_params(p, accumulate);
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     const int elem = bf16 ? 2 : 4;
     k.vecs = p->C * elem / 16;
@@ -1337,8 +1348,10 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     // super-block: as many sub-blocks as keep the whole height range in one chunk (<= 8 cells: larger
     // ones pack the geometry lanes better but leave too few warps to overlap geometry with gathers)
     int sbx = (p->tune[3] >> 4) & 0xf, sby = (p->tune[3] >> 8) & 0xf;
-    if (k.out_bf16) {
-        sbx = sby = 1;  // a rounded output cannot take partial sums: keep the accumulators in registers
+    if (k.out_bf16 || k.accumulate) {
+        // a rounded output cannot take partial sums, and an output that already holds another level's result
+        // must be added once, at the end: keep the accumulators in registers
+        sbx = sby = 1;
     } else if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
         sbx = sby = 1;
         while (true) {
@@ -1383,13 +1396,13 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     return FLASHBEV_OK;
 }
 
-flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
+flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false)
 {
     KParams k;
     int V, warps;
     dim3 grid;
     size_t smem;
-    const flashbev_status st = configure_tiled(p, k, V, warps, grid, smem);
+    const flashbev_status st = configure_tiled(p, k, V, warps, grid, smem, accumulate);
     if (st != FLASHBEV_OK) return st;
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     cudaError_t e;
@@ -1408,12 +1421,12 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream)
     return e == cudaSuccess ? FLASHBEV_OK : FLASHBEV_CUDA_ERROR;
 }
 
-flashbev_status run_device(const flashbev_vt_params *p, cudaStream_t stream)
+flashbev_status run_device(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false)
 {
     flashbev_status st;
     const bool tiled = p->kernel == FLASHBEV_KERNEL_TILED || (p->kernel == FLASHBEV_KERNEL_AUTO && tiled_applicable(p));
     if (tiled && !tiled_applicable(p)) return FLASHBEV_UNSUPPORTED;
-    st = tiled ? launch_tiled(p, stream) : launch_per_output(p, stream);
+    st = tiled ? launch_tiled(p, stream, accumulate) : launch_per_output(p, stream, accumulate);
     if (st != FLASHBEV_OK) return st;
     if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
     t_last_launches = 1;
@@ -1543,6 +1556,33 @@ flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params 
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
     t_last_launches = 1;
     t_last_kernel = V == 1 ? "tiled_bwd_v1" : (V == 2 ? "tiled_bwd_v2" : "tiled_bwd_v4");
+    return FLASHBEV_OK;
+}
+
+// ---- multi-resolution gathering: one launch per pyramid level, levels after the first add to the output
+flashbev_status flashbev_sampling_vt_multires(const flashbev_vt_multires_params *q, void *stream)
+{
+    if (!q || q->struct_size < sizeof(flashbev_vt_multires_params) || !q->base || !q->features || !q->feat_hw)
+        return FLASHBEV_INVALID_ARG;
+    if (q->levels < 1 || q->levels > FLASHBEV_MAX_LEVELS) return FLASHBEV_INVALID_ARG;
+    if (q->base->struct_size < sizeof(flashbev_vt_params)) return FLASHBEV_INVALID_ARG;
+    flashbev_vt_params lv[FLASHBEV_MAX_LEVELS];
+    flashbev_status st;
+    for (int l = 0; l < q->levels; ++l) {  // every level is checked before anything is enqueued
+        lv[l] = *q->base;
+        lv[l].struct_size = sizeof(flashbev_vt_params);
+        lv[l].features = q->features[l];
+        lv[l].feat_h = q->feat_hw[2 * l], lv[l].feat_w = q->feat_hw[2 * l + 1];
+        if (l > 0) lv[l].valid_count_out = nullptr;
+        if (!params_ok(&lv[l], st)) return st;
+        if (lv[l].out_dtype != FLASHBEV_F32) return FLASHBEV_UNSUPPORTED;
+        if ((st = check_alignment(&lv[l])) != FLASHBEV_OK) return st;
+        const bool tiled = lv[l].kernel == FLASHBEV_KERNEL_TILED;
+        if (tiled && !tiled_applicable(&lv[l])) return FLASHBEV_UNSUPPORTED;
+    }
+    for (int l = 0; l < q->levels; ++l)
+        if ((st = run_device(&lv[l], static_cast<cudaStream_t>(stream), l > 0)) != FLASHBEV_OK) return st;
+    t_last_launches = q->levels;
     return FLASHBEV_OK;
 }
 

@@ -226,3 +226,22 @@ def make_sca_inputs(P=8, X=200, Y=200, seed=0):
     weights = (e / e.sum(-1, keepdims=True)).reshape(1, Q, heads, len(levels), P).astype(np.float32)
     return dict(value=value, level_hw=np.array(levels, np.int32), lidar2img=mats, offsets=offsets, weights=weights,
                 img_hw=img_hw, bev_range=(-51.2, 51.2, -51.2, 51.2, -5.0, 3.0), grid=(X, Y, Zref))
+
+
+def make_pyramid_inputs(w: Workload, levels: int = 3, stream: int = 0):
+    """A feature pyramid for the multi-resolution variant: level l has the map of `w` halved l times
+    (rounded up), the same cameras and channel count, independent standard-normal values.
+    Returns (list of Inputs-like feature arrays [B,N,Hf_l,Wf_l,C] float32, list of bf16 bit arrays or None, lidar2img)."""
+    base = make_inputs(w, stream)
+    rng = rng_for(w.index, 900 + stream)
+    feats, bits = [base.features], [base.features_bf16]
+    Hf, Wf = w.feat_hw
+    for _ in range(1, levels):
+        Hf, Wf = (Hf + 1) // 2, (Wf + 1) // 2
+        f = rng.standard_normal((w.B, w.N, Hf, Wf, w.C), dtype=np.float32)
+        b = None
+        if w.dtype == "bf16":
+            f, b = round_to_bf16(f)
+        feats.append(f)
+        bits.append(b)
+    return feats, bits, base.lidar2img

@@ -288,11 +288,13 @@ def measure_tensorized(torch, w, device, iters=5):
     return {"latency_ms": a.elapsed_time(b) / iters, "peak_mb": (torch.cuda.max_memory_allocated() - base) / 1e6}
 
 
-def measure_sca(torch, device, P, iters=10, chunk_records=0):
+def measure_sca(torch, device, P, iters=10, chunk_records=0, bf16=False):
     """Latency of the fused spatial cross-attention at BEVFormer-base sizes (inputs ~350 MB+ per call: L2-cold)."""
     from paper_2607_10071_b200 import binding as fb
     c = wl.make_sca_inputs(P=P)
     t = {k: torch.from_numpy(c[k]).to(device) for k in ("value", "lidar2img", "offsets", "weights")}
+    if bf16:
+        t["value"] = t["value"].to(torch.bfloat16)
     out = torch.empty((1, c["grid"][0] * c["grid"][1], 256), dtype=torch.float32, device=device)
     call = lambda: fb.sca(t["value"], c["level_hw"], t["lidar2img"], t["offsets"], t["weights"], c["img_hw"],
                           c["bev_range"], c["grid"], out=out, chunk_records=chunk_records)
@@ -305,7 +307,7 @@ def measure_sca(torch, device, P, iters=10, chunk_records=0):
         call()
     b.record()
     torch.cuda.synchronize()
-    bytes_unique = sum(v.numel() * 4 for v in t.values()) + out.numel() * 4
+    bytes_unique = sum(v.numel() * v.element_size() for v in t.values()) + out.numel() * 4
     ms = a.elapsed_time(b) / iters
     return {"latency_ms": ms, "unique_mb": bytes_unique / 1e6, "hbm_roofline_frac_of_measured":
             bytes_unique / (ms * 1e-3) / 1e9 / measured_peaks()[0]}
@@ -460,6 +462,7 @@ def main():
             f"P={P}": dict(measure_sca(torch, device, P), paper_flashsca_ms=ms, paper_bevformer_sca_ms=base,
                            paper_hardware="RTX 4070 Ti SUPER, TensorRT FP32 (Table 7)")
             for P, ms, base in ((8, 5.27, 8.96), (16, 8.16, 15.81), (32, 13.90, 29.27))}
+        context["flashsca_bevformer_base"]["P=8, bf16 values"] = measure_sca(torch, device, 8, bf16=True)
         context["representative_backward_latency_ms"] = measure_backward(
             torch, w if w.name == "representative" else wl.get("representative"), args, device,
             max(3, args.steps // 4), 3, barrier)

@@ -213,13 +213,15 @@ typedef struct flashbev_sca_params {
     size_t struct_size;        /* sizeof(flashbev_sca_params) of the caller's header */
     const void *value;         /* device, [B][N][T][heads][head_dim], T = sum_l H_l*W_l (levels concatenated,
                                   each level row-major); value_dtype, 16-byte aligned */
-    int32_t value_dtype;       /* FLASHBEV_F32 (bf16 values: FLASHBEV_UNSUPPORTED) */
+    int32_t value_dtype;       /* FLASHBEV_F32 or FLASHBEV_BF16 (accumulation and output are float32 either way) */
     int32_t chunk_records;     /* tuning: tap records built per pass over a query (shared memory per warp); 0 = default */
     const int32_t *level_hw;   /* HOST, [L][2] = (H_l, W_l); read during the call only; L <= 8 */
     const float *lidar2img;    /* device, [B][N][4][4] float32 */
     const float *offsets;      /* device, [B][X*Y][heads][L][P][2] float32, in texels of level l */
     const float *weights;      /* device, [B][X*Y][heads][L][P] float32 (normally a softmax over L*P) */
-    int32_t B, N, heads, head_dim; /* head_dim a multiple of 4, <= 128; heads * head_dim / 4 <= 128 lanes x 4 */
+    int32_t B, N, heads, head_dim; /* head_dim a multiple of 4 (float32) or 8 (bfloat16), <= 128; a head's
+                                      16-byte vectors must divide 32, at most 4 (float32) / 2 (bfloat16)
+                                      passes of 32 lanes over the heads: else FLASHBEV_UNSUPPORTED */
     int32_t L, P;
     int32_t img_h, img_w;
     double x_min, x_max;

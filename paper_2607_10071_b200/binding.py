@@ -274,14 +274,16 @@ def flashbev_sca(params: ScaParams, stream: int | None = None, check: bool = Tru
 
 def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, out=None, hits=None, stream=None,
         chunk_records=0):
-    """value: CUDA float32 [B,N,T,heads,Dh]; offsets [B,Q,heads,L,P,2]; weights [B,Q,heads,L,P] (CUDA float32).
+    """value: CUDA float32 or bfloat16 [B,N,T,heads,Dh]; offsets [B,Q,heads,L,P,2]; weights [B,Q,heads,L,P] (CUDA float32).
     level_hw: sequence of (H_l, W_l).  Returns CUDA float32 [B, Q, heads*Dh] (marshalling only)."""
     import numpy as np
     import torch
 
-    for t in (value, lidar2img, offsets, weights):
+    for t in (lidar2img, offsets, weights):
         if not t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
             raise ValueError("sca needs contiguous CUDA float32 tensors")
+    if not value.is_cuda or not value.is_contiguous() or value.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("value must be a contiguous CUDA float32 or bfloat16 tensor")
     B, N, T, heads, Dh = value.shape
     X, Y, Zref = grid
     L, P = weights.shape[3], weights.shape[4]
@@ -290,7 +292,8 @@ def sca(value, level_hw, lidar2img, offsets, weights, img_hw, bev_range, grid, o
         out = torch.empty((B, X * Y, heads * Dh), dtype=torch.float32, device=value.device)
     p = ScaParams()
     p.struct_size = ctypes.sizeof(ScaParams)
-    p.value, p.value_dtype, p.chunk_records = value.data_ptr(), F32, int(chunk_records)
+    p.value, p.chunk_records = value.data_ptr(), int(chunk_records)
+    p.value_dtype = F32 if value.dtype == torch.float32 else BF16
     p.level_hw = lv.ctypes.data
     p.lidar2img, p.offsets, p.weights = lidar2img.data_ptr(), offsets.data_ptr(), weights.data_ptr()
     p.B, p.N, p.heads, p.head_dim, p.L, p.P = B, N, heads, Dh, L, P

@@ -918,11 +918,11 @@ constexpr int kScaMaxLevels = 8;
 constexpr int kScaMaxChunkPoints = 32;  // sampling points per chunk (bit mask of visible points)
 
 struct ScaParams {
-    const float4 *value;   // [B][N][T][D / 4]
+    const uint4 *value;    // [B][N][T][16-byte vectors of the D channels], float32 or bfloat16
     const float *l2i;
     const float2 *offsets; // [B][Q][heads][L][P]
     const float *weights;  // [B][Q][heads][L][P]
-    float4 *out;           // [B][Q][D / 4]
+    float4 *out;           // [B][Q][D / 4], float32
     int32_t *hits_out;
     int B, N, heads, Dh, L, P, X, Y, Zref, Himg, Wimg;
     int lph, hp;           // lanes per head, heads per pass
@@ -957,7 +957,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 __device__ __forceinline__ int small_div(int i, float inv) { return (int)(((float)i + 0.5f) * inv); }
 
 // EVEN: every lane has a head in every pass (heads = V * heads per pass, 32 lanes all used)
-template <int V, bool EVEN>
+template <int V, bool EVEN, bool BF16>
 __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -1033,17 +1033,19 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
 
     // ---- lanes -> (head, 16-byte slice of the head's channels)
     const int hsub = lane / p.lph, e4 = lane - hsub * p.lph;
-    float2 acc[V][2];
+    constexpr int PV = BF16 ? 4 : 2;  // channel pairs per 16-byte vector
+    float2 acc[V][PV];
     bool on[V];
     int hrow[V];  // first record of the lane's head
 #pragma unroll
     for (int v = 0; v < V; ++v) {
-        acc[v][0] = acc[v][1] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
         const int h = v * p.hp + hsub;
         on[v] = EVEN || (hsub < p.hp && h < p.heads);
         hrow[v] = (on[v] ? h : 0) * p.pitch;
     }
-    const int D4 = p.heads * p.lph;  // float4 per texel
+    const int D4 = p.heads * p.lph;  // 16-byte vectors per texel
     const int nbase = p.Zref * p.L;
 
     for (int pt0 = 0, c = 0; pt0 < p.P; pt0 += p.Pc, ++c) {
@@ -1066,7 +1068,7 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
             // visible points of the chunk: the reference height a point belongs to must be seen
             const uint32_t vis = __ballot_sync(FULL, lane < npc && ((mask >> klane) & 1u));
             if (vis == 0u) continue;
-            const uint4 *vcam = reinterpret_cast<const uint4 *>(p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4) + e4;
+            const uint4 *vcam = p.value + ((size_t)b * p.N + n) * (size_t)p.T * D4 + e4;
             __syncwarp();  // the previous records and reference positions have been consumed
             // texel position of every visible reference on every level: integer part and fraction
             for (int e = lane; e < nbase; e += 32) {
@@ -1140,10 +1142,10 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
                         if (!on[v]) continue;
-                        fma_vec<false>(acc[v], s[v][0], make_float2(tw[v].x, tw[v].x));
-                        fma_vec<false>(acc[v], s[v][1], make_float2(tw[v].y, tw[v].y));
-                        fma_vec<false>(acc[v], s[v][2], make_float2(tw[v].z, tw[v].z));
-                        fma_vec<false>(acc[v], s[v][3], make_float2(tw[v].w, tw[v].w));
+                        fma_vec<BF16>(acc[v], s[v][0], make_float2(tw[v].x, tw[v].x));
+                        fma_vec<BF16>(acc[v], s[v][1], make_float2(tw[v].y, tw[v].y));
+                        fma_vec<BF16>(acc[v], s[v][2], make_float2(tw[v].z, tw[v].z));
+                        fma_vec<BF16>(acc[v], s[v][3], make_float2(tw[v].w, tw[v].w));
                     }
                 }
             }
@@ -1153,8 +1155,11 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         if (!on[v]) continue;
-        __stcs(p.out + ((size_t)b * Q + q) * D4 + (v * p.hp + hsub) * p.lph + e4,
-               make_float4(acc[v][0].x * g, acc[v][0].y * g, acc[v][1].x * g, acc[v][1].y * g));
+        // the lane's 16-byte vector of values is PV / 2 float4 of output
+        float4 *o = p.out + (((size_t)b * Q + q) * D4 + (v * p.hp + hsub) * p.lph + e4) * (PV / 2);
+#pragma unroll
+        for (int e = 0; e < PV; e += 2)
+            __stcs(o + e / 2, make_float4(acc[v][e].x * g, acc[v][e].y * g, acc[v][e + 1].x * g, acc[v][e + 1].y * g));
     }
     if (p.hits_out && lane == 0) p.hits_out[gq] = hits;
 }
@@ -1605,17 +1610,19 @@ flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
         k.Hl[l] = Hl, k.Wl[l] = Wl, k.lvl0[l] = (int)T;
         T += (long long)Hl * Wl;
     }
-    if (q->value_dtype != FLASHBEV_F32 || q->L > kScaMaxLevels || q->N > kMaxCams || q->Zref > 32) return FLASHBEV_UNSUPPORTED;
-    if (q->head_dim % 4 || q->head_dim > 128 || (long long)q->N * q->Zref > 1024) return FLASHBEV_UNSUPPORTED;
+    const bool bf16 = q->value_dtype == FLASHBEV_BF16;
+    const int epv = bf16 ? 8 : 4;  // elements per 16-byte vector
+    if (q->L > kScaMaxLevels || q->N > kMaxCams || q->Zref > 32) return FLASHBEV_UNSUPPORTED;
+    if (q->head_dim % epv || q->head_dim > 128 || (long long)q->N * q->Zref > 1024) return FLASHBEV_UNSUPPORTED;
     if (T >= 2147483647LL || (double)q->B * q->X * q->Y >= 2147483648.0) return FLASHBEV_UNSUPPORTED;
     if (((uintptr_t)q->value % 16) || ((uintptr_t)q->out % 16) || ((uintptr_t)q->offsets % 8) ||
         ((uintptr_t)q->weights % 4) || ((uintptr_t)q->lidar2img % 4) || (q->hits_out && ((uintptr_t)q->hits_out % 4)))
         return FLASHBEV_MISALIGNED;
-    k.lph = q->head_dim / 4;
+    k.lph = q->head_dim / epv;
     k.hp = 32 / k.lph;
     const int V = (q->heads + k.hp - 1) / k.hp;
     if (V > 4) return FLASHBEV_UNSUPPORTED;
-    k.value = static_cast<const float4 *>(q->value);
+    k.value = static_cast<const uint4 *>(q->value);
     k.l2i = q->lidar2img;
     k.offsets = reinterpret_cast<const float2 *>(q->offsets);
     k.weights = q->weights;
@@ -1648,13 +1655,19 @@ flashbev_status flashbev_sca(const flashbev_sca_params *q, void *stream_)
     };
     cudaError_t e;
     const bool even = k.hp * k.lph == 32 && q->heads == V * k.hp;
-    if (V == 1) e = even ? launch(sca_kernel<1, true>) : launch(sca_kernel<1, false>);
-    else if (V == 2) e = even ? launch(sca_kernel<2, true>) : launch(sca_kernel<2, false>);
-    else if (V == 3) e = even ? launch(sca_kernel<3, true>) : launch(sca_kernel<3, false>);
-    else e = even ? launch(sca_kernel<4, true>) : launch(sca_kernel<4, false>);
+    if (bf16) {
+        if (V == 1) e = even ? launch(sca_kernel<1, true, true>) : launch(sca_kernel<1, false, true>);
+        else if (V == 2) e = even ? launch(sca_kernel<2, true, true>) : launch(sca_kernel<2, false, true>);
+        else return FLASHBEV_UNSUPPORTED;
+    } else {
+        if (V == 1) e = even ? launch(sca_kernel<1, true, false>) : launch(sca_kernel<1, false, false>);
+        else if (V == 2) e = even ? launch(sca_kernel<2, true, false>) : launch(sca_kernel<2, false, false>);
+        else if (V == 3) e = even ? launch(sca_kernel<3, true, false>) : launch(sca_kernel<3, false, false>);
+        else e = even ? launch(sca_kernel<4, true, false>) : launch(sca_kernel<4, false, false>);
+    }
     if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
     t_last_launches = 1;
-    t_last_kernel = "sca_f32";
+    t_last_kernel = bf16 ? "sca_bf16" : "sca_f32";
     return FLASHBEV_OK;
 }
 

@@ -13,10 +13,13 @@ from tests.test_oracle_sca_pins import make_case
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(c):
+def run_gpu(c, bf16=False):
     import torch
     dev = torch.device("cuda:0")
     t = {k: torch.from_numpy(np.ascontiguousarray(c[k])).to(dev) for k in ("value", "lidar2img", "offsets", "weights")}
+    if bf16:  # c["value"] already holds bf16-representable numbers; ship their 16-bit patterns
+        bits = wl.round_to_bf16(c["value"])[1]
+        t["value"] = torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
     B = c["value"].shape[0]
     Q = c["grid"][0] * c["grid"][1]
     D = c["value"].shape[3] * c["value"].shape[4]
@@ -24,14 +27,16 @@ def run_gpu(c):
     hits = torch.full((B, Q), -1, dtype=torch.int32, device=dev)
     fb.sca(t["value"], c["level_hw"], t["lidar2img"], t["offsets"], t["weights"], c["img_hw"], c["bev_range"], c["grid"],
            out=out, hits=hits)
-    assert fb.flashbev_last_kernel_name() == "sca_f32" and fb.flashbev_last_launch_count() == 1
+    assert fb.flashbev_last_kernel_name() == ("sca_bf16" if bf16 else "sca_f32") and fb.flashbev_last_launch_count() == 1
     torch.cuda.synchronize()
     return out.cpu().numpy(), hits.cpu().numpy()
 
 
-def check(oracle, c, label=""):
+def check(oracle, c, label="", bf16=False):
+    if bf16:  # the oracle sees the same bf16-rounded values the kernel reads
+        c = dict(c, value=wl.round_to_bf16(c["value"])[0])
     ref, rhits, flagged = oracle.sca(**c)
-    out, hits = run_gpu(c)
+    out, hits = run_gpu(c, bf16)
     assert np.all(np.isfinite(out)), label
     keep = flagged == 0
     assert np.array_equal(hits[keep], rhits[keep]), label
@@ -58,6 +63,26 @@ def test_point_and_level_counts(oracle, P, Zref, L):
     check(oracle, c, f"P={P} Zref={Zref} L={L}")
 
 
+@pytest.mark.parametrize("general", [False, True])
+@pytest.mark.parametrize("heads,Dh", [(8, 32), (4, 8), (2, 16), (1, 128), (3, 24), (16, 16), (16, 8), (40, 8)])
+def test_bf16_values(oracle, general, heads, Dh):
+    """bfloat16 value maps, fp32 accumulation: the only error left is the summation order."""
+    c = make_case(heads * 100 + Dh + 7, B=2, N=6, heads=heads, Dh=Dh, levels=((12, 18), (6, 9), (3, 5)), P=4,
+                  grid=(9, 7, 2), general=general, rng_xy=10.0)
+    check(oracle, c, f"bf16 heads={heads} Dh={Dh}", bf16=True)
+
+
+def test_bf16_unsupported_shapes():
+    import torch
+    c = make_case(5, N=2, heads=2, Dh=4, grid=(4, 4, 2))
+    dev = torch.device("cuda:0")
+    t = {k: torch.from_numpy(np.ascontiguousarray(c[k])).to(dev) for k in ("value", "lidar2img", "offsets", "weights")}
+    with pytest.raises(fb.FlashBevError) as e:   # head_dim 4 is half a 16-byte vector of bfloat16
+        fb.sca(t["value"].to(torch.bfloat16), c["level_hw"], t["lidar2img"], t["offsets"], t["weights"], c["img_hw"],
+               c["bev_range"], c["grid"])
+    assert e.value.status == fb.UNSUPPORTED
+
+
 def test_non_finite_and_unseen(oracle):
     c = make_case(3, N=4, heads=2, Dh=4, grid=(6, 6, 2))
     c["lidar2img"][0, 1, 0, 2] = np.nan
@@ -74,3 +99,4 @@ def test_bevformer_base_shape(oracle):
     """N = 6, C = 256, 8 heads, 200 x 200 queries, Zref = 4, L = 4, P = 8 (the paper's Table 7 setting), ring rig."""
     c = wl.make_sca_inputs(P=8)
     print("\n" + check(oracle, c, "bevformer-base P=8"))
+    print(check(oracle, c, "bevformer-base P=8, bf16 values", bf16=True))

@@ -57,6 +57,7 @@ struct KParams {
     int lcap;                   // records per cell list
     int slots;                  // record slots per warp
     int wcap;                   // walker descriptors per warp and height chunk
+    int wide;                   // host side: use the instance with adjacent channel vectors and 256-bit loads
 };
 
 // ------------------------------------------------------------------------------------------
@@ -551,10 +552,18 @@ __device__ __forceinline__ void fma_vec(float2 (&acc)[BF16 ? 4 : 2], const uint4
     }
 }
 
+// Two adjacent 16-byte vectors with one 256-bit load (sm_100: ld.global.v8), 32-byte aligned address.
+__device__ __forceinline__ void ldg_pair(const uint4 *ptr, uint4 &a, uint4 &b)
+{
+    asm("ld.global.nc.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+        : "l"(ptr));
+}
+
 // Gather of one cell list by its channel lanes, U records per iteration.  Every record is two
 // taps of one texel row, both always loadable.  Lanes whose list is shorter than the warp's
 // longest repeat their last record with weight 0; lanes with no records do nothing.
-template <int V, bool BF16>
+template <int V, bool BF16, bool WIDE>
 __device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int4 *list, int nrec, int maxn,
                                             const uint4 *const (&featv)[V])
 {
@@ -566,13 +575,23 @@ __device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], cons
 #pragma unroll
         for (int u = 0; u < U; ++u) r[u] = list[min(j + u, last)];
         uint4 t[U][2][V];
+        if (WIDE) {  // the lane's vectors are adjacent: V / 2 loads of 32 bytes per tap
 #pragma unroll
-        for (int u = 0; u < U; ++u)
+            for (int u = 0; u < U; ++u)
 #pragma unroll
-            for (int v = 0; v < V; ++v) {
-                t[u][0][v] = __ldg(featv[v] + r[u].x);
-                t[u][1][v] = __ldg(featv[v] + r[u].y);
-            }
+                for (int v = 0; v + 1 < V; v += 2) {
+                    ldg_pair(featv[v] + r[u].x, t[u][0][v], t[u][0][v + 1]);
+                    ldg_pair(featv[v] + r[u].y, t[u][1][v], t[u][1][v + 1]);
+                }
+        } else {
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    t[u][0][v] = __ldg(featv[v] + r[u].x);
+                    t[u][1][v] = __ldg(featv[v] + r[u].y);
+                }
+        }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const bool has = j + u <= last;
@@ -605,7 +624,8 @@ __device__ __forceinline__ void scatter_list(const float4 (&go)[V], const bool (
     }
 }
 
-template <int V, bool BF16, int WARPS, bool BWD>
+// WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
+template <int V, bool BF16, int WARPS, bool BWD, bool WIDE>
 __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 20 : 24)) / WARPS)
     vt_tiled_kernel(const KParams p)
 {
@@ -659,7 +679,9 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
     // ---- gather role of this lane inside a sub-block
     const int cg = lane / p.g, gl = lane - cg * p.g;
     const bool role = cg < p.cpw;
-    const int vec0 = blockIdx.y * (p.g * V) + gl;  // first channel vector of this lane
+    constexpr bool kWide = WIDE && V >= 2 && !BWD;
+    const int vstep = kWide ? 1 : p.g;  // distance between the lane's channel vectors
+    const int vec0 = kWide ? (blockIdx.y * p.g + gl) * V : blockIdx.y * (p.g * V) + gl;  // the lane's first vector
     // channel vectors past the end of the row (ragged last channel block) re-read vector 0, never stored
     const uint4 *featv[V];
     float4 *gfv[V];  // backward: where this lane's channel vectors of a texel's gradient live
@@ -667,7 +689,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
         const size_t cam0 = (size_t)b * p.N * p.Hf * p.Wf * p.vecs;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
-            const int vi = (vec0 + v * p.g < p.vecs) ? vec0 + v * p.g : 0;
+            const int vi = (vec0 + v * vstep < p.vecs) ? vec0 + v * vstep : 0;
             featv[v] = BWD ? nullptr : static_cast<const uint4 *>(p.feat) + cam0 + vi;
             gfv[v] = BWD ? reinterpret_cast<float4 *>(p.gfeat) + cam0 + vi : nullptr;
         }
@@ -826,7 +848,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                             bool on[V];
 #pragma unroll
                             for (int v = 0; v < V; ++v) {
-                                const int vi = vec0 + v * p.g;
+                                const int vi = vec0 + v * vstep;
                                 go[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                                 on[v] = vi < p.vecs;
                                 if (on[v]) {
@@ -844,7 +866,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
 #pragma unroll
                             for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
                     }
-                    gather_list<V, BF16>(acc, sm.list + cell * (p.lcap + 1), nrec, maxn, featv);
+                    gather_list<V, BF16, kWide>(acc, sm.list + cell * (p.lcap + 1), nrec, maxn, featv);
                     const bool stored = (touched >> s) & 1u;
                     // one sub-block per warp: accumulators live on; several: add to the stored partial sums
                     const bool write = lane_on && (p.sbn > 1 ? (nrec > 0 || (final && (!stored ||
@@ -858,7 +880,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 2
                         float *o = p.out + ocell * p.C;
 #pragma unroll
                         for (int v = 0; v < V; ++v) {
-                            const int vi = vec0 + v * p.g;
+                            const int vi = vec0 + v * vstep;
                             if (vi < p.vecs) {
 #pragma unroll
                                 for (int e = 0; e < PV; e += 2) {
@@ -1292,15 +1314,15 @@ bool tiled_applicable(const flashbev_vt_params *p)
     return vecs_total < 2147483648.0;
 }
 
-template <int V, bool BF16, int WARPS, bool BWD>
+template <int V, bool BF16, int WARPS, bool BWD, bool WIDE = false>
 cudaError_t launch_tiled_inst(const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
 {
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    vt_tiled_kernel<V, BF16, WARPS, BWD><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
+    vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
     return cudaSuccess;
 }
 
@@ -1311,7 +1333,9 @@ cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t sm
         case 1: return launch_tiled_inst<V, BF16, 1, false>(k, grid, smem, stream);
         case 2: return launch_tiled_inst<V, BF16, 2, false>(k, grid, smem, stream);
         case 8: return launch_tiled_inst<V, BF16, 8, false>(k, grid, smem, stream);
-        default: return launch_tiled_inst<V, BF16, 4, false>(k, grid, smem, stream);
+        default:
+            if (V >= 2 && k.wide) return launch_tiled_inst<V, BF16, 4, false, (V >= 2)>(k, grid, smem, stream);
+            return launch_tiled_inst<V, BF16, 4, false>(k, grid, smem, stream);
     }
 }
 
@@ -1329,7 +1353,9 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     int g = p->tune[1];
     if (!(V == 1 || V == 2 || V == 4) || g < 1 || g > 32) V = 0, g = 0;
     if (!V) {
-        if (k.vecs <= 8) V = 1, g = k.vecs;
+        // tall columns: the geometry of a column dominates, eight cells per sub-block amortise it better
+        if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
+        else if (k.vecs <= 8) V = 1, g = k.vecs;
         else if (k.vecs <= 16) V = (k.vecs % 2 == 0) ? 2 : 1, g = (k.vecs + V - 1) / V;
         else if (k.vecs <= 64) V = 2, g = (k.vecs + 1) / 2;
         else V = 4, g = (k.vecs + 3) / 4;
@@ -1396,6 +1422,10 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     const int cblocks = (k.vecs + g * V - 1) / (g * V);
     if (ctas > 2147483647LL || cblocks > 65535 || p->B > 65535) return FLASHBEV_UNSUPPORTED;
     grid = dim3((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
+    // adjacent vectors and 256-bit loads: half the load instructions (bf16 features are issue-bound), and whole
+    // texels per cell where the strided 16-byte segments of a cell would not cover whole 128-byte lines
+    k.wide = warps == 4 && V >= 2 && k.vecs % V == 0 && (uintptr_t)p->features % 32 == 0 &&
+             (bf16 || (g * 16) % 128 != 0) && !(p->tune[3] & 0x10000);
     smem = align16(cta_table_bytes(p->N)) +
                         (size_t)warps * warp_smem_layout(nullptr, nullptr, k.ct, k.slots, k.zc, k.wcap);
     return FLASHBEV_OK;

@@ -88,3 +88,20 @@ def test_bf16_output_with_nchw(oracle):
     out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, SUM, layout=fb.NCHW, out_dtype=fb.BF16)
     got = _bf16_to_f32(out.permute(0, 2, 3, 1)).astype(np.float64)
     assert np.all(np.abs(got - ref.out) <= 1e-4 + np.abs(ref.out) * 2.0 ** -8)
+
+
+@pytest.mark.parametrize("name", ["representative", "half_taller"])
+def test_feature_pointer_aligned_to_16_but_not_32_bytes(name):
+    """The 256-bit loads need 32-byte alignment; a tensor that starts 16 bytes later takes the 128-bit
+    instance and must give the same numbers (every cell adds its taps in the same order)."""
+    import torch
+    w = wl.get(name)
+    inp = wl.make_inputs(w)
+    f, m = _cuda_features(inp, fb.NHWC)
+    shifted_store = torch.empty(f.numel() + 16 // f.element_size(), dtype=f.dtype, device=f.device)
+    shifted = shifted_store[16 // f.element_size():].view(f.shape)
+    shifted.copy_(f)
+    assert f.data_ptr() % 32 == 0 and shifted.data_ptr() % 32 == 16
+    a = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, w.reduce)
+    b = fb.sampling_vt(shifted, m, w.img_hw, w.bev_range, w.grid, w.reduce)
+    assert torch.equal(a, b)

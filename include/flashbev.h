@@ -108,7 +108,8 @@ typedef struct flashbev_vt_params {
     int32_t *valid_count_out;  /* optional [B][X][Y] int32: sum_z sum_n M_n per cell; NULL to skip */
     int32_t tune[4];           /* 0 = library defaults.  tune[0]: channel vectors per lane (1,2,4);
                                   tune[1]: lanes per cell; tune[2]: height bins per geometry walker;
-                                  tune[3]: bits 0-3 warps per CTA (1,2,4,8), bits 4-7 / 8-11 sub-blocks per warp in x / y.
+                                  tune[3]: bits 0-3 warps per CTA (1,2,4,8), bits 4-7 / 8-11 sub-blocks per warp in x / y,
+                                  bits 12-15 super-blocks per warp, bit 16 never / bit 17 always use 256-bit feature loads.
                                   Invalid values fall back to the defaults */
 } flashbev_vt_params;
 

@@ -1357,8 +1357,8 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
         if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
         else if (k.vecs <= 8) V = 1, g = k.vecs;
         else if (k.vecs <= 16) V = (k.vecs % 2 == 0) ? 2 : 1, g = (k.vecs + V - 1) / V;
-        else if (k.vecs <= 64) V = 2, g = (k.vecs + 1) / 2;
-        else V = 4, g = (k.vecs + 3) / 4;
+        else if (k.vecs < 24) V = 2, g = (k.vecs + 1) / 2;
+        else V = 4, g = (k.vecs + 3) / 4;  // wide texels: four vectors per lane keep 2-5 cells in a sub-block
         if (g > 32) g = 32;
     }
     warps = p->tune[3] & 0xf;
@@ -1424,8 +1424,8 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     grid = dim3((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
     // adjacent vectors and 256-bit loads: half the load instructions (bf16 features are issue-bound), and whole
     // texels per cell where the strided 16-byte segments of a cell would not cover whole 128-byte lines
-    k.wide = warps == 4 && V >= 2 && k.vecs % V == 0 && (uintptr_t)p->features % 32 == 0 &&
-             (bf16 || (g * 16) % 128 != 0) && !(p->tune[3] & 0x10000);
+    k.wide = warps == 4 && (V == 2 || (V == 4 && (p->tune[3] & 0x20000))) && k.vecs % V == 0 && (uintptr_t)p->features % 32 == 0 &&
+             (bf16 || (g * 16) % 128 != 0 || (p->tune[3] & 0x20000)) && !(p->tune[3] & 0x10000);
     smem = align16(cta_table_bytes(p->N)) +
                         (size_t)warps * warp_smem_layout(nullptr, nullptr, k.ct, k.slots, k.zc, k.wcap);
     return FLASHBEV_OK;

@@ -975,9 +975,6 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// i / n for 0 <= i < 2^20, given inv = 1 / n in fp32
-__device__ __forceinline__ int small_div(int i, float inv) { return (int)(((float)i + 0.5f) * inv); }
-
 // EVEN: every lane has a head in every pass (heads = V * heads per pass, 32 lanes all used)
 template <int V, bool EVEN, bool BF16>
 __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParams p)

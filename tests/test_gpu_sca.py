@@ -13,7 +13,7 @@ from tests.test_oracle_sca_pins import make_case
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(c, bf16=False):
+def run_gpu(c, bf16=False, chunk_records=0):
     import torch
     dev = torch.device("cuda:0")
     t = {k: torch.from_numpy(np.ascontiguousarray(c[k])).to(dev) for k in ("value", "lidar2img", "offsets", "weights")}
@@ -26,17 +26,17 @@ def run_gpu(c, bf16=False):
     out = torch.full((B, Q, D), float("nan"), dtype=torch.float32, device=dev)
     hits = torch.full((B, Q), -1, dtype=torch.int32, device=dev)
     fb.sca(t["value"], c["level_hw"], t["lidar2img"], t["offsets"], t["weights"], c["img_hw"], c["bev_range"], c["grid"],
-           out=out, hits=hits)
+           out=out, hits=hits, chunk_records=chunk_records)
     assert fb.flashbev_last_kernel_name() == ("sca_bf16" if bf16 else "sca_f32") and fb.flashbev_last_launch_count() == 1
     torch.cuda.synchronize()
     return out.cpu().numpy(), hits.cpu().numpy()
 
 
-def check(oracle, c, label="", bf16=False):
+def check(oracle, c, label="", bf16=False, chunk_records=0):
     if bf16:  # the oracle sees the same bf16-rounded values the kernel reads
         c = dict(c, value=wl.round_to_bf16(c["value"])[0])
     ref, rhits, flagged = oracle.sca(**c)
-    out, hits = run_gpu(c, bf16)
+    out, hits = run_gpu(c, bf16, chunk_records)
     assert np.all(np.isfinite(out)), label
     keep = flagged == 0
     assert np.array_equal(hits[keep], rhits[keep]), label
@@ -81,6 +81,14 @@ def test_bf16_unsupported_shapes():
         fb.sca(t["value"].to(torch.bfloat16), c["level_hw"], t["lidar2img"], t["offsets"], t["weights"], c["img_hw"],
                c["bev_range"], c["grid"])
     assert e.value.status == fb.UNSUPPORTED
+
+
+@pytest.mark.parametrize("P,Zref,records", [(5, 4, 16), (7, 3, 24), (12, 4, 64), (9, 2, 8), (33, 4, 0)])
+def test_ragged_point_chunks(oracle, P, Zref, records):
+    """Points are processed in chunks of `records / (heads * L)`: last chunks that are shorter, chunks that
+    do not start on a multiple of Zref, one point per chunk, and more than 32 points."""
+    c = make_case(P * 100 + Zref, N=6, heads=4, Dh=8, levels=((16, 24), (8, 12)), P=P, grid=(8, 9, Zref), rng_xy=12.0)
+    check(oracle, c, f"P={P} Zref={Zref} records={records}", chunk_records=records)
 
 
 def test_non_finite_and_unseen(oracle):

@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 def cases(draw):
     dtype = draw(st.sampled_from(["f32", "bf16"]))
     vec = 4 if dtype == "f32" else 8
-    C = vec * draw(st.integers(1, 12)) if draw(st.booleans()) else draw(st.integers(1, 40))
+    C = vec * draw(st.sampled_from([1, 2, 3, 5, 8, 9, 12, 16, 20, 23, 24, 27, 32, 40, 66])) if draw(st.booleans()) else draw(st.integers(1, 40))
     return dict(
         seed=draw(st.integers(0, 10_000)), dtype=dtype, C=C,
         B=draw(st.integers(1, 2)), N=draw(st.integers(1, 7)),
@@ -25,7 +25,7 @@ def cases(draw):
         walk=draw(st.sampled_from([0, 1, 3, 8])))
 
 
-@settings(max_examples=40, deadline=None, derandomize=True,
+@settings(max_examples=60, deadline=None, derandomize=True,
           suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
 @given(case=cases())
 def test_random_small_problems_match_the_oracle(oracle, case):

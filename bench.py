@@ -239,6 +239,43 @@ def measure_workload(torch, w, args, device, rank, dist_barrier, steps, warmup, 
             "kernel": kname, "df": df}
 
 
+def measure_regimes(torch, df, device):
+    """Secondary figures of one workload, from the frames already on the device: warm-L2 latency (the same frame
+    back to back in a graph), the latency of single launches without a graph (events around each launch, frames
+    rotating, so L2-cold), and the number of valid samples (from the kernel's own count output)."""
+    fb = df.fb
+    w = df.w
+    X, Y, Z = w.grid
+    stream = torch.cuda.Stream(device)
+    reps = 20
+    with torch.cuda.stream(stream):
+        sp = stream.cuda_stream
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(reps):
+                fb.flashbev_sampling_vt(df.params[0], torch.cuda.current_stream().cuda_stream)
+        _, per = time_steps(torch, graph.replay, 10, 3, lambda: None)
+        warm = statistics.median(per) / reps
+        singles = []
+        for _ in range(3):
+            for p in df.params:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fb.flashbev_sampling_vt(p, sp)
+                b.record()
+                singles.append((a, b))
+        torch.cuda.synchronize()
+        single = statistics.median(a.elapsed_time(b) for a, b in singles[len(df.params):])
+        cnt = torch.zeros((w.B, X, Y), dtype=torch.int32, device=device)
+        pc = fb.make_params(df.feats[0].data_ptr(), fb.BF16 if w.dtype == "bf16" else fb.F32, df.mats[0].data_ptr(),
+                            w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid, w.reduce, df.outs[0].data_ptr(),
+                            cnt.data_ptr())
+        fb.flashbev_sampling_vt(pc, sp)
+        torch.cuda.synchronize()
+    return {"warm_l2_latency_ms": round(warm, 5), "single_launch_no_graph_latency_ms": round(single, 5),
+            "valid_samples": int(cnt.sum().item())}
+
+
 def measure_backward(torch, w, args, device, steps, warmup, dist_barrier):
     """Latency of flashbev_sampling_vt_backward (memset + scatter kernel) per frame, L2-cold frames."""
     from paper_2607_10071_b200 import binding as fb
@@ -433,10 +470,13 @@ def main():
         for name in wl.CONFIG_ORDER:
             wi = wl.get(name)
             mi = measure_workload(torch, wi, args, device, rank, barrier, max(3, args.steps // 4), 3)
-            mi.pop("df")
+            extra = measure_regimes(torch, mi.pop("df"), device)
             lat = statistics.mean(mi["per_step_ms"]) / mi["frames"]
             peak, _ = measured_peaks()
             table[name] = {"latency_ms": round(lat, 5), "sample_channels_per_s": wi.sample_channels / (lat * 1e-3),
+                           "latency_ms_median": round(statistics.median(mi["per_step_ms"]) / mi["frames"], 5),
+                           "latency_ms_min": round(min(mi["per_step_ms"]) / mi["frames"], 5),
+                           "valid_sample_channels_per_s": extra["valid_samples"] * wi.C / (lat * 1e-3), **extra,
                            "hbm_roofline_frac_of_measured": wi.unique_bytes / (lat * 1e-3) / 1e9 / peak,
                            "hbm_roofline_frac_of_8TBs": wi.unique_bytes / (lat * 1e-3) / 1e9 / 8000.0,
                            "unique_mb": round(wi.unique_bytes / 1e6, 3), "output_mb": round(wi.output_bytes / 1e6, 3),

@@ -43,7 +43,8 @@ def test_binding_exposes_the_same_names():
 
 @pytest.mark.parametrize("cname,mirror", [("flashbev_vt_params", "VtParams"),
                                           ("flashbev_vt_backward_params", "VtBackwardParams"),
-                                          ("flashbev_sca_params", "ScaParams")])
+                                          ("flashbev_sca_params", "ScaParams"),
+                                          ("flashbev_vt_multires_params", "VtMultiresParams")])
 def test_ctypes_struct_matches_the_c_struct(tmp_path, cname, mirror):
     prog = tmp_path / "layout.c"
     cls = getattr(fb, mirror)
@@ -113,6 +114,48 @@ def test_host_entry_validates_staging():
     assert fb.flashbev_sampling_vt_host(p, 4096 + 8, need, None, check=False) == fb.MISALIGNED
     assert fb.flashbev_sampling_vt_host(p, 4096, need - 1, None, check=False) == fb.TOO_SMALL
     assert fb.flashbev_workspace_bytes(p) == 0
+
+
+def test_multires_arguments_are_validated_on_the_host():
+    """Level count, null levels and map sizes are checked before any CUDA call (fake, aligned addresses)."""
+    base = good_params()
+    hw = [(16, 44), (8, 22)]
+    ptrs = [4096, 8192]
+    assert fb.flashbev_sampling_vt_multires(base, [], [], None, check=False) == fb.INVALID_ARG
+    assert fb.flashbev_sampling_vt_multires(base, ptrs * 5, hw * 5, None, check=False) == fb.INVALID_ARG
+    assert fb.flashbev_sampling_vt_multires(base, [4096, 0], hw, None, check=False) == fb.INVALID_ARG
+    assert fb.flashbev_sampling_vt_multires(base, ptrs, [(16, 44), (0, 22)], None, check=False) == fb.INVALID_ARG
+    assert fb.flashbev_sampling_vt_multires(base, [4096, 8192 + 2], hw, None, check=False) == fb.MISALIGNED
+    assert fb.flashbev_sampling_vt_multires(good_params(out_dtype=fb.BF16), ptrs, hw, None, check=False) == fb.UNSUPPORTED
+    assert fb.lib().flashbev_sampling_vt_multires(None, None) == fb.INVALID_ARG
+
+
+def test_sca_arguments_are_validated_on_the_host():
+    import numpy as np
+    lv = np.array([[4, 6], [2, 3]], np.int32)
+
+    def params(**over):
+        p = fb.ScaParams()
+        p.struct_size = ctypes.sizeof(fb.ScaParams)
+        p.value, p.value_dtype, p.level_hw = 4096, fb.F32, lv.ctypes.data
+        p.lidar2img, p.offsets, p.weights, p.out = 8192, 12288, 16384, 20480
+        p.B, p.N, p.heads, p.head_dim, p.L, p.P = 1, 2, 2, 8, 2, 4
+        p.img_h, p.img_w = 32, 48
+        p.x_min, p.x_max, p.y_min, p.y_max, p.z_min, p.z_max = -1, 1, -1, 1, -1, 1
+        p.X, p.Y, p.Zref = 3, 3, 2
+        for k, v in over.items():
+            setattr(p, k, v)
+        return p
+
+    for over, status in [(dict(value=None), fb.INVALID_ARG), (dict(heads=0), fb.INVALID_ARG), (dict(P=0), fb.INVALID_ARG),
+                         (dict(x_max=-1.0), fb.INVALID_ARG), (dict(value_dtype=7), fb.INVALID_ARG),
+                         (dict(chunk_records=-1), fb.INVALID_ARG), (dict(head_dim=6), fb.UNSUPPORTED),
+                         (dict(head_dim=132), fb.UNSUPPORTED), (dict(Zref=33), fb.UNSUPPORTED),
+                         (dict(value_dtype=fb.BF16, head_dim=4), fb.UNSUPPORTED), (dict(heads=200), fb.UNSUPPORTED),
+                         (dict(value=4096 + 4), fb.MISALIGNED), (dict(offsets=12288 + 4), fb.MISALIGNED),
+                         (dict(struct_size=8), fb.INVALID_ARG)]:
+        assert fb.flashbev_sca(params(**over), None, check=False) == status, over
+    assert fb.lib().flashbev_sca(None, None) == fb.INVALID_ARG
 
 
 def test_product_path_never_imports_the_oracle():

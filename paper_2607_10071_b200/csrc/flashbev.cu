@@ -1370,11 +1370,15 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     if (k.cpw == 5 || k.cpw == 7) k.wy = k.cpw;
     k.wx = k.cpw / k.wy;
     k.cpw = k.wx * k.wy;
-    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : (p->Z <= 16 ? 4 : (p->Z <= 32 ? 8 : 16));
+    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : (p->Z < 16 ? 4 : (p->Z <= 32 ? 8 : 16));
     const int runs = (p->Z + k.walk - 1) / k.walk;  // walkers per column when all of Z is one chunk
 
     // super-block: as many sub-blocks as keep the whole height range in one chunk (<= 8 cells: larger
     // ones pack the geometry lanes better but leave too few warps to overlap geometry with gathers)
+    // record slots per warp: 16 and more height bins write long lists, and every list that fills up costs another
+    // walk-and-gather round (measured: 64 bins, 8 cells: 128 slots 458 us, 384 slots 368 us, 512 slots 399 us;
+    // 16 bins, 8 cells: 192 slots 172 us, 384 slots 162 us, 512 slots 173 us -- shared memory then costs warps)
+    const int slot_budget = p->Z >= 16 ? 384 : 192;
     int sbx = (p->tune[3] >> 4) & 0xf, sby = (p->tune[3] >> 8) & 0xf;
     if (k.out_bf16 || k.accumulate) {
         // a rounded output cannot take partial sums, and an output that already holds another level's result
@@ -1383,11 +1387,11 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     } else if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
         sbx = sby = 1;
         while (true) {
-            const bool grow_x = sbx * k.wx <= sby * k.wy;
+            const bool grow_x = sbx * k.wx < sby * k.wy;  // square so far: grow along y, the contiguous output axis
             const int nx = grow_x ? sbx * 2 : sbx, ny = grow_x ? sby : sby * 2;
             const int ct = nx * ny * k.cpw;
             // keep the whole height range in one chunk and leave each cell a list of ~1.5 Z + 4 records
-            if (ct > 8 || (long long)ct * p->N * runs > 512 || 2 * ct * (3 * p->Z + 8) > 2 * 2 * 192) break;
+            if (ct > 8 || (long long)ct * p->N * runs > 512 || ct * (3 * p->Z / 2 + 4) > slot_budget) break;
             // small problems: rather one warp per sub-block than idle SMs (a warp's latency is the kernel's)
             if ((long long)p->B * p->X * p->Y / ct < (long long)sm_count() * 24) break;
             sbx = nx, sby = ny;
@@ -1401,9 +1405,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     k.band = 4;
     k.reps = (p->tune[3] >> 12) & 0xf;
     if (k.reps < 1) k.reps = 1;
-    // record slots per warp: tall columns write long lists, and every list that fills up costs another
-    // walk-and-gather round (measured on 64 bins: 128 slots 458 us, 384 slots 368 us, 512 slots 399 us)
-    k.slots = std::max(k.sbn > 1 ? 192 : 128, k.ct * std::min(48, 3 * p->Z / 4));
+    k.slots = p->Z >= 16 ? slot_budget : (k.sbn > 1 ? 192 : 128);
     k.lcap = k.slots / k.ct;
     // height chunk: all walkers of a chunk must fit the warp's descriptor array
     k.wcap = (int)std::min<long long>(512, std::max<long long>(128, (long long)k.ct * p->N * runs));

@@ -1387,7 +1387,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     } else if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
         sbx = sby = 1;
         while (true) {
-            const bool grow_x = sbx * k.wx < sby * k.wy;  // square so far: grow along y, the contiguous output axis
+            const bool grow_x = sby > sbx;  // first along y, the contiguous output axis (1-2 % on three of four shapes)
             const int nx = grow_x ? sbx * 2 : sbx, ny = grow_x ? sby : sby * 2;
             const int ct = nx * ny * k.cpw;
             // keep the whole height range in one chunk and leave each cell a list of ~1.5 Z + 4 records

@@ -37,7 +37,7 @@ from paper_2607_10071_b200 import workloads as wl  # noqa: E402
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (bytes; None where no capture of that workload exists)
-NCU_DRAM_TRAFFIC = {"representative": 4.76e6, "long_range": 47.31e6}
+NCU_DRAM_TRAFFIC = {"representative": 4.76e6, "long_range": 42.40e6}
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "fused_sampling_vt_throughput"
 UNIT = "sample-channels/s"

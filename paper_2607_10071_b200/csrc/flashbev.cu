@@ -1,6 +1,7 @@
 // Fused Sampling-VT for B200 (sm_100a): kernels and the C ABI declared in flashbev.h.
 //
-// Two kernels compute the same operator (paper Eq. 1, fused as in Algorithm 2):
+// Two kernels compute the same operator (paper Eq. 1, fused as in Algorithm 2); a third, at the end of the
+// kernel part, is the fused spatial cross-attention of Sec. 4.4:
 //
 //   vt_per_output_kernel  one thread per (cell, channel group); every thread recomputes the
 //                         projection of every (z, n) itself.  This is the work decomposition
@@ -13,7 +14,7 @@
 //                         in fp64 and turned into a compact list of row records in shared
 //                         memory; successive heights that land on the same texel rows are merged
 //                         into one record before any feature is touched.  Channel lanes then walk
-//                         the list with 128-bit loads and fp32 FMAs.  Nothing but the output is
+//                         the list with 128- or 256-bit loads and fp32 FMAs.  Nothing but the output is
 //                         written to global memory.
 //
 // Geometry (projection, validity, floor, fractions) is fp64, weights and accumulation fp32.
@@ -282,7 +283,7 @@ __global__ void __launch_bounds__(256) vt_per_output_nchw_kernel(const KParams p
 //       busy over the ct * N columns), split into short runs ("walkers");
 //   (B) walkers: a lane follows a run with exact fp64 geometry and merges successive bins that
 //       land on the same texel rows into row records in the cell's shared-memory list;
-//   (C) gather, one sub-block at a time: channel lanes walk their cell's list with 128-bit loads
+//   (C) gather, one sub-block at a time: channel lanes walk their cell's list with 128- or 256-bit loads
 //       and packed fp32 FMAs, then store.
 // Warps of a CTA share only the per-batch-element tables staged once at kernel start, so while
 // one warp is in its geometry another streams features.

@@ -1355,7 +1355,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
         if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
         else if (k.vecs <= 8) V = 1, g = k.vecs;
         else if (k.vecs <= 16) V = (k.vecs % 2 == 0) ? 2 : 1, g = (k.vecs + V - 1) / V;
-        else if (k.vecs < 24) V = 2, g = (k.vecs + 1) / 2;
+        else if (k.vecs < 24 || (k.vecs <= 32 && p->Z >= 16)) V = 2, g = (k.vecs + 1) / 2;  // (16+ bins: 0-17 % over V = 4)
         else V = 4, g = (k.vecs + 3) / 4;  // wide texels: four vectors per lane keep 2-5 cells in a sub-block
         if (g > 32) g = 32;
     }

@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 SOURCES = [os.path.join(_HERE, "csrc", "flashbev.cu")]
-HEADERS = [os.path.join(ROOT, "include", "flashbev.h")]
+HEADERS = [os.path.join(ROOT, "include", "flashbev.h"), os.path.join(_HERE, "csrc", "vt_tiled.cuh")]
 LIB = os.path.join(_HERE, "libflashbev.so")
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

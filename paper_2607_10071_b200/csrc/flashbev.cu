@@ -47,18 +47,17 @@ struct KParams {
     // tiled kernel only
     int vecs;                   // 16-byte vectors per texel (C * elem / 16)
     int g;                      // lanes per cell
-    int cpw;                    // cells per sub-block (= wx * wy): the cells one gather pass covers
+    int cpw;                    // cells per sub-block (= wx * wy <= 8): the cells one warp works on at a time
     int wx, wy;                 // sub-block size in cells (x, y)
-    int sbx, sby, sbn;          // sub-blocks per super-block (x, y, total)
-    int ct, ct_inv;             // cells per super-block (<= 32) and ceil(65536 / ct)
-    int blocks_x, blocks_y;     // super-blocks per batch element
-    int band, reps;             // super-block order: bands of `band` rows; super-blocks per warp
-    int zc;                     // height bins per chunk (multiple of 4 unless == Z)
-    int walk;                   // height bins per walker
-    int lcap;                   // records per cell list
-    int slots;                  // record slots per warp
-    int wcap;                   // walker descriptors per warp and height chunk
+    int blocks_x, blocks_y;     // sub-blocks per batch element
+    int band, reps;             // sub-block order: bands of `band` rows; sub-blocks per warp
+    int slots;                  // record slots per warp (>= 64)
+    int ncap;                   // column descriptors per warp (= cpw * N)
+    int den_bytes;              // bytes of the per-(cell, height) camera counts per warp (Eq. 1 mode, else 0)
+    int rstep;                  // distance (16-byte vectors) from a record's first tap to its second: vecs, or 0 on 1-texel-wide maps
+    int nvec_cam;               // N * Hf * Wf * vecs: vectors of one batch element's feature maps (bounds-checked build)
     int wide;                   // host side: use the instance with adjacent channel vectors and 256-bit loads
+    unsigned *err;              // bounds-checked build: device word that counts out-of-range indices (may be null)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -73,6 +72,24 @@ __device__ __forceinline__ double fast_rcp(double d)
     e = fma(-d, r, 1.0);
     return fma(r, e, r);
 }
+
+// Index guard.  In the bounds-checked build (-DFLASHBEV_DEBUG_BOUNDS) every computed shared-memory slot, record
+// offset and output index of the tiled kernel goes through this: an index outside [0, n) is counted into the
+// caller's device word and replaced by 0, so the access that follows stays in range.  In the normal build it
+// is the identity and costs nothing.
+#ifdef FLASHBEV_DEBUG_BOUNDS
+__device__ __forceinline__ int fb_idx(long long i, long long n, unsigned *err)
+{
+    if (i < 0 || i >= n) {
+        if (err) atomicAdd(err, 1u);
+        return 0;
+    }
+    return (int)i;
+}
+#define FB_IDX(i, n, err) fb_idx((long long)(i), (long long)(n), (err))
+#else
+#define FB_IDX(i, n, err) (i)
+#endif
 
 struct Sample {
     int x0, y0;
@@ -276,652 +293,8 @@ __global__ void __launch_bounds__(256) vt_per_output_nchw_kernel(const KParams p
 }
 
 // ------------------------------------------------------------------------------------------
-// Kernel 2: tiled.  Every WARP owns a super-block of adjacent BEV cells (ct <= 32 cells, made of
-// sbn sub-blocks of cpw cells) and takes it through three phases on its own, synchronising only
-// with __syncwarp:
-//   (A) per (cell, camera) column: the interval of height bins that can be valid (all 32 lanes
-//       busy over the ct * N columns), split into short runs ("walkers");
-//   (B) walkers: a lane follows a run with exact fp64 geometry and merges successive bins that
-//       land on the same texel rows into row records in the cell's shared-memory list;
-//   (C) gather, one sub-block at a time: channel lanes walk their cell's list with 128- or 256-bit loads
-//       and packed fp32 FMAs, then store.
-// Warps of a CTA share only the per-batch-element tables staged once at kernel start, so while
-// one warp is in its geometry another streams features.
-//
-// A list that fills up makes its walkers stop; the warp then gathers what it has and runs another
-// round.  With one sub-block per warp the accumulators simply stay in registers across rounds and
-// height chunks; with several, a sub-block's partial sums are added to its own output elements
-// (owner-only read-modify-write, no atomics) and the last round applies the normalisation.
-//
-// Shared memory (dynamic):
-//   CTA   : double mats[N][12]   rows 0..2 of lidar2img[b][n], rows 0/1 pre-scaled to feature px
-//           float  slope[N][5]   per camera: d/dk of the five validity conditions
-//           int    celltab[32]   position of cell c inside a super-block: lx | ly << 8
-//   warp  : int4    list[slots + ct]  per cell lcap (+1 pad) records {offL, offR, wL, wR}
-//           double2 cellxy[32]   voxel-centre (x_w, y_w) of the cells (NaN: outside the grid)
-//           uint32  walkers[wcap] packed (cell, camera, first bin in chunk, bins - 1)
-//           uint32  den[ct * zc / 4] per (cell, z) camera counts, one byte each (Eq. 1 mode)
-//           uint32  wsave[9][32] state of a walker that stopped because its list was full
-//           int     list_count[32], list_end[32], cell_count[32], n_walkers
-
-constexpr int kSaveWords = 9;
-constexpr int kWalkIlp = 4;  // height bins whose geometry a walker evaluates independently
-
-struct WarpSmem {
-    int4 *list;
-    double2 *cellxy;
-    uint32_t *walkers;
-    uint32_t *den;
-    uint32_t *wsave;
-    int *list_count;
-    int *list_end;
-    int *cell_count;
-    int *n_walkers;
-};
-
-__host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t)15; }
-
-__host__ __device__ inline size_t cta_table_bytes(int N)
-{
-    return align16((size_t)N * 12 * sizeof(double)) + align16((size_t)N * 5 * sizeof(float)) + 32 * sizeof(int);
-}
-
-__host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem *t, int ct, int slots, int zc, int wcap)
-{
-    size_t o = 0;
-    auto take = [&](size_t bytes) {
-        unsigned char *ptr = base ? base + o : nullptr;
-        o += align16(bytes);
-        return ptr;
-    };
-    unsigned char *p0 = take((size_t)(slots + ct) * sizeof(int4));
-    unsigned char *p1 = take((size_t)32 * sizeof(double2));
-    unsigned char *p2 = take((size_t)wcap * sizeof(uint32_t));
-    unsigned char *p3 = take((size_t)((ct * zc + 3) / 4) * sizeof(uint32_t));
-    unsigned char *p4 = take((size_t)kSaveWords * 32 * sizeof(uint32_t));
-    unsigned char *p5 = take((size_t)(3 * 32 + 4) * sizeof(int));
-    if (t) {
-        t->list = reinterpret_cast<int4 *>(p0);
-        t->cellxy = reinterpret_cast<double2 *>(p1);
-        t->walkers = reinterpret_cast<uint32_t *>(p2);
-        t->den = reinterpret_cast<uint32_t *>(p3);
-        t->wsave = reinterpret_cast<uint32_t *>(p4);
-        t->list_count = reinterpret_cast<int *>(p5);
-        t->list_end = t->list_count + 32;
-        t->cell_count = t->list_end + 32;
-        t->n_walkers = t->cell_count + 32;
-    }
-    return o;
-}
-
-// Exact (fp64) test and bilinear set-up of height bin k of a (cell, camera) column:
-// row_i(z) = a_i + m[4 i + 2] * z_w.  When the camera's depth row does not depend on z
-// (m[10] == 0: no pitch or roll) 1/d is computed once per column.
-struct ColumnWalk {
-    const double *m;
-    double a0, a1, a2, zc0, dz, wlim, hlim, rconst;
-    bool dconst, dead;
-
-    __device__ __forceinline__ void init(const KParams &p, const double *mats, int n, double2 xy)
-    {
-        m = mats + n * 12;
-        a0 = fma(m[1], xy.y, fma(m[0], xy.x, m[3]));
-        a1 = fma(m[5], xy.y, fma(m[4], xy.x, m[7]));
-        a2 = fma(m[9], xy.y, fma(m[8], xy.x, m[11]));
-        zc0 = p.z_min + 0.5 * p.dz;
-        dz = p.dz;
-        wlim = (double)p.Wf - 0.5;
-        hlim = (double)p.Hf - 0.5;
-        dconst = (m[10] == 0.0);
-        dead = dconst && !(a2 > kDepthMin);
-        rconst = (dconst && !dead) ? fast_rcp(a2) : 0.0;
-    }
-    // Branch-free apart from the (warp-uniform in practice) choice of the reciprocal.
-    __device__ __forceinline__ bool sample(int k, Sample &s) const
-    {
-        const double zw = fma((double)k, dz, zc0);
-        const double d = dconst ? a2 : fma(m[10], zw, a2);
-        const double r = dconst ? rconst : fast_rcp(d);  // d <= 0 or NaN gives inf/NaN: every test below fails
-        const double fx = fma(fma(m[2], zw, a0), r, -0.5);
-        const double fy = fma(fma(m[6], zw, a1), r, -0.5);
-        const double flx = floor(fx), fly = floor(fy);
-        s.x0 = (int)flx;
-        s.y0 = (int)fly;
-        s.tx = (float)(fx - flx);
-        s.ty = (float)(fy - fly);
-        return (d > kDepthMin) & (fx > -0.5) & (fx < wlim) & (fy > -0.5) & (fy < hlim);
-    }
-};
-
-// Walker state: the two open texel rows (oy, oy + 1) at column ox with their merged weights.
-struct Walker {
-    int k, ox, oy, vcount;
-    bool open;
-    float uL, uR, lL, lR;
-
-    // Close rows and write them as records.  False (nothing changed) if the list is full.
-    __device__ __forceinline__ bool close_rows(const KParams &p, const WarpSmem &sm, int wc, int wn, int4 *wlist,
-                                               bool close_u, bool close_l)
-    {
-        // A tap outside the map gets weight 0 and the address of the record's other tap.
-        const bool inL = ox >= 0, inR = ox + 1 <= p.Wf - 1;
-        const float cuL = inL ? uL : 0.f, cuR = inR ? uR : 0.f;
-        const float clL = inL ? lL : 0.f, clR = inR ? lR : 0.f;
-        const bool emit_u = close_u && oy >= 0 && oy <= p.Hf - 1 && (cuL != 0.f || cuR != 0.f);
-        const bool emit_l = close_l && oy + 1 >= 0 && oy + 1 <= p.Hf - 1 && (clL != 0.f || clR != 0.f);
-        const int need = (int)emit_u + (int)emit_l;
-        if (!need) return true;
-        const int slot = atomicAdd(&sm.list_count[wc], need);
-        if (slot >= p.lcap) {  // full (one pad slot lets a 2-record write start at lcap - 1)
-            atomicMin(&sm.list_end[wc], slot);
-            return false;
-        }
-        const int rowv = p.Wf * p.vecs;
-        const int o = ((wn * p.Hf + oy) * p.Wf + ox) * p.vecs;
-        const int oL = inL ? o : o + p.vecs, oR = inR ? o + p.vecs : o;
-        int sl = slot;
-        if (emit_u) wlist[sl++] = make_int4(oL, oR, __float_as_int(cuL), __float_as_int(cuR));
-        if (emit_l) wlist[sl] = make_int4(oL + rowv, oR + rowv, __float_as_int(clL), __float_as_int(clR));
-        return true;
-    }
-
-    // Add one valid sample.  False (nothing changed) if a row had to be written and the list is full.
-    // keep: same two rows; down / up: moved by one row, one open row is carried over.
-    __device__ __forceinline__ bool add(const KParams &p, const WarpSmem &sm, int wc, int wn, int4 *wlist,
-                                        const Sample &s, float scale)
-    {
-        const bool same_col = open & (s.x0 == ox);
-        const int dy = s.y0 - oy;
-        const bool keep = same_col & (dy == 0), down = same_col & (dy == 1), up = same_col & (dy == -1);
-        const bool close_u = open & !(keep | up), close_l = open & !(keep | down);
-        if (close_u | close_l) {
-            if (!close_rows(p, sm, wc, wn, wlist, close_u, close_l)) return false;
-        }
-        const float wx1 = s.tx, wx0 = 1.f - s.tx;
-        const float wy1 = s.ty * scale, wy0 = (1.f - s.ty) * scale;
-        const float w00 = wx0 * wy0, w01 = wx1 * wy0, w10 = wx0 * wy1, w11 = wx1 * wy1;
-        const float nuL = w00 + (keep ? uL : (down ? lL : 0.f)), nuR = w01 + (keep ? uR : (down ? lR : 0.f));
-        const float nlL = w10 + (keep ? lL : (up ? uL : 0.f)), nlR = w11 + (keep ? lR : (up ? uR : 0.f));
-        uL = nuL, uR = nuR, lL = nlL, lR = nlR;
-        open = true;
-        ox = s.x0;
-        oy = s.y0;
-        ++vcount;
-        return true;
-    }
-};
-
-// Runs a walker from its saved position to the end of its run.  False if it had to stop.
-__device__ __forceinline__ bool run_walker(const KParams &p, const WarpSmem &sm, const double *mats, Walker &w, int wc,
-                                           int wn, int kend, int kc0, int4 *wlist)
-{
-    ColumnWalk cw;
-    cw.init(p, mats, wn, sm.cellxy[wc]);
-    while (w.k <= kend) {
-        Sample s[kWalkIlp];
-        bool ok[kWalkIlp];
-#pragma unroll
-        for (int i = 0; i < kWalkIlp; ++i) ok[i] = (w.k + i <= kend) && cw.sample(w.k + i, s[i]);
-#pragma unroll
-        for (int i = 0; i < kWalkIlp; ++i) {
-            if (ok[i]) {
-                float scale = 1.f;
-                if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
-                    const int di = wc * p.zc + (w.k + i - kc0);
-                    const uint32_t dn = (sm.den[di >> 2] >> (8 * (di & 3))) & 0xffu;
-                    scale = 1.f / (float)(dn > 1u ? dn : 1u);
-                }
-                if (!w.add(p, sm, wc, wn, wlist, s[i], scale)) {
-                    w.k += i;
-                    return false;
-                }
-            }
-        }
-        w.k += kWalkIlp;
-    }
-    if (w.open) {
-        if (!w.close_rows(p, sm, wc, wn, wlist, true, true)) return false;
-        w.open = false;
-    }
-    return true;
-}
-
-// Phase A: per (cell, camera) column of the super-block, a conservative interval of height bins of
-// the chunk [kc0, kc1) that can be valid (every validity condition is linear in z once d > 0),
-// split into walkers of at most p.walk bins.
-__device__ __forceinline__ void phase_a(const KParams &p, const WarpSmem &sm, const double *mats, const float *slope,
-                                        unsigned in_mask, int kc0, int kc1, int lane)
-{
-    for (int pr = lane; pr < p.ct * p.N; pr += 32) {
-        const int n = (pr * p.ct_inv) >> 16, c = pr - n * p.ct;
-        if (!((in_mask >> c) & 1u)) continue;
-        const double2 xy = sm.cellxy[c];
-        const double *m = mats + n * 12;
-        const float *sl = slope + n * 5;
-        const double zc0 = p.z_min + 0.5 * p.dz;  // centre of bin 0; z_w(k) = zc0 + k dz
-        // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom
-        const double d0 = fma(m[10], zc0, fma(m[9], xy.y, fma(m[8], xy.x, m[11])));
-        float lo = (float)kc0 - 1.f, hi = (float)kc1;
-        bool empty = false;
-        auto cond = [&](float a, float bslope) {
-            if (bslope > 0.f) lo = fmaxf(lo, -a * __frcp_rn(bslope));       // k > -a/b
-            else if (bslope < 0.f) hi = fminf(hi, -a * __frcp_rn(bslope));  // k < -a/b
-            else if (a <= 0.f) empty = true;  // independent of z (NaN: keep, tested exactly later)
-        };
-        cond((float)(d0 - kDepthMin), sl[0]);
-        if (empty || !(lo < hi)) continue;
-        const double p00 = fma(m[2], zc0, fma(m[1], xy.y, fma(m[0], xy.x, m[3])));
-        cond((float)p00, sl[1]);
-        cond((float)fma((double)p.Wf, d0, -p00), sl[2]);
-        if (empty || !(lo < hi)) continue;
-        const double p10 = fma(m[6], zc0, fma(m[5], xy.y, fma(m[4], xy.x, m[7])));
-        cond((float)p10, sl[3]);
-        cond((float)fma((double)p.Hf, d0, -p10), sl[4]);
-        if (empty) continue;
-        // widen by a guard far above the float error; every bin is re-tested exactly later
-        const float guard = 0.05f + 1e-5f * (float)p.Z;
-        int klo = (int)floorf(fminf(fmaxf(lo - guard, (float)kc0 - 1.f), (float)kc1)) + 1;
-        int khi = (int)ceilf(fmaxf(fminf(hi + guard, (float)kc1), (float)kc0 - 1.f)) - 1;
-        klo = max(klo, kc0);
-        khi = min(khi, kc1 - 1);
-        if (klo > khi) continue;
-        const int nw = (khi - klo + p.walk) / p.walk;
-        const int base = atomicAdd(sm.n_walkers, nw);
-        for (int i = 0; i < nw; ++i) {
-            const int k0 = klo + i * p.walk, k1 = min(khi, k0 + p.walk - 1);
-            if (base + i < p.wcap)
-                sm.walkers[base + i] = (uint32_t)c | ((uint32_t)n << 8) | ((uint32_t)(k0 - kc0) << 14) |
-                                       ((uint32_t)(k1 - k0) << 23);
-        }
-    }
-}
-
-// acc += w * (channels of one 16-byte vector), two channels per packed fp32 FMA
-template <bool BF16>
-__device__ __forceinline__ void fma_vec(float2 (&acc)[BF16 ? 4 : 2], const uint4 &t, const float2 w)
-{
-    if (BF16) {
-        acc[0] = __ffma2_rn(make_float2(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u)), w, acc[0]);
-        acc[1] = __ffma2_rn(make_float2(__uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u)), w, acc[1]);
-        acc[2 % (BF16 ? 4 : 2)] =
-            __ffma2_rn(make_float2(__uint_as_float(t.z << 16), __uint_as_float(t.z & 0xffff0000u)), w, acc[2 % (BF16 ? 4 : 2)]);
-        acc[3 % (BF16 ? 4 : 2)] =
-            __ffma2_rn(make_float2(__uint_as_float(t.w << 16), __uint_as_float(t.w & 0xffff0000u)), w, acc[3 % (BF16 ? 4 : 2)]);
-    } else {
-        acc[0] = __ffma2_rn(make_float2(__uint_as_float(t.x), __uint_as_float(t.y)), w, acc[0]);
-        acc[1] = __ffma2_rn(make_float2(__uint_as_float(t.z), __uint_as_float(t.w)), w, acc[1]);
-    }
-}
-
-// Two adjacent 16-byte vectors with one 256-bit load (sm_100: ld.global.v8), 32-byte aligned address.
-__device__ __forceinline__ void ldg_pair(const uint4 *ptr, uint4 &a, uint4 &b)
-{
-    asm("ld.global.nc.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-        : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
-        : "l"(ptr));
-}
-
-// Gather of one cell list by its channel lanes, U records per iteration.  Every record is two
-// taps of one texel row, both always loadable.  Lanes whose list is shorter than the warp's
-// longest repeat their last record with weight 0; lanes with no records do nothing.
-template <int V, bool BF16, bool WIDE>
-__device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int4 *list, int nrec, int maxn,
-                                            const uint4 *const (&featv)[V])
-{
-    constexpr int U = V == 1 ? 4 : (V == 2 ? (BF16 ? 3 : 2) : 1);  // measured: bf16 gains 2 % from the third record
-    if (nrec <= 0) return;
-    const int last = nrec - 1;
-    for (int j = 0; j < maxn; j += U) {
-        int4 r[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) r[u] = list[min(j + u, last)];
-        uint4 t[U][2][V];
-        if (WIDE) {  // the lane's vectors are adjacent: V / 2 loads of 32 bytes per tap
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int v = 0; v + 1 < V; v += 2) {
-                    ldg_pair(featv[v] + r[u].x, t[u][0][v], t[u][0][v + 1]);
-                    ldg_pair(featv[v] + r[u].y, t[u][1][v], t[u][1][v + 1]);
-                }
-        } else {
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    t[u][0][v] = __ldg(featv[v] + r[u].x);
-                    t[u][1][v] = __ldg(featv[v] + r[u].y);
-                }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const bool has = j + u <= last;
-            const float wl = has ? __int_as_float(r[u].z) : 0.f;
-            const float wr = has ? __int_as_float(r[u].w) : 0.f;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                fma_vec<BF16>(acc[v], t[u][0][v], make_float2(wl, wl));
-                fma_vec<BF16>(acc[v], t[u][1][v], make_float2(wr, wr));
-            }
-        }
-    }
-}
-
-// Backward of the gather: every record adds its two weighted taps of the cell's output gradient to
-// the feature gradient (the transpose of gather_list).  Vector atomics: texels are shared by cells.
-template <int V>
-__device__ __forceinline__ void scatter_list(const float4 (&go)[V], const bool (&on)[V], const int4 *list, int nrec,
-                                             float4 *const (&gfv)[V])
-{
-    for (int j = 0; j < nrec; ++j) {
-        const int4 r = list[j];
-        const float wl = __int_as_float(r.z), wr = __int_as_float(r.w);
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            if (!on[v]) continue;  // ragged last channel block
-            if (wl != 0.f) atomicAdd(gfv[v] + r.x, make_float4(go[v].x * wl, go[v].y * wl, go[v].z * wl, go[v].w * wl));
-            if (wr != 0.f) atomicAdd(gfv[v] + r.y, make_float4(go[v].x * wr, go[v].y * wr, go[v].z * wr, go[v].w * wr));
-        }
-    }
-}
-
-// WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
-template <int V, bool BF16, int WARPS, bool BWD, bool WIDE>
-__global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : 20) / WARPS)
-    vt_tiled_kernel(const KParams p)
-{
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    constexpr int PV = BF16 ? 4 : 2;  // channel pairs per 16-byte vector
-    constexpr int THREADS = WARPS * 32;
-    constexpr unsigned FULL = 0xffffffffu;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.z;
-
-    double *mats = reinterpret_cast<double *>(smem_raw);
-    float *slope = reinterpret_cast<float *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)));
-    int *celltab = reinterpret_cast<int *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)) +
-                                           align16((size_t)p.N * 5 * sizeof(float)));
-    WarpSmem sm;
-    {
-        const size_t per_warp = warp_smem_layout(nullptr, nullptr, p.ct, p.slots, p.zc, p.wcap);
-        warp_smem_layout(smem_raw + align16(cta_table_bytes(p.N)) + warp * per_warp, &sm, p.ct, p.slots, p.zc, p.wcap);
-    }
-
-    // ---- per-CTA tables: camera matrices (scaled to feature px), condition slopes, cell positions
-    for (int i = tid; i < p.N * 12; i += THREADS) {
-        const int n = i / 12, e = i - n * 12;
-        double v = (double)__ldg(p.l2i + ((size_t)b * p.N + n) * 16 + e);
-        if (e < 4) v *= p.sx;
-        else if (e < 8) v *= p.sy;
-        mats[i] = v;
-    }
-    for (int n = tid; n < p.N; n += THREADS) {
-        const float *M = p.l2i + ((size_t)b * p.N + n) * 16;
-        const double m2 = (double)__ldg(M + 2) * p.sx, m6 = (double)__ldg(M + 6) * p.sy, m10 = (double)__ldg(M + 10);
-        // d/dk of: depth - 0.1, p0s, Wf d - p0s, p1s, Hf d - p1s
-        slope[n * 5 + 0] = (float)(m10 * p.dz);
-        slope[n * 5 + 1] = (float)(m2 * p.dz);
-        slope[n * 5 + 2] = (float)(((double)p.Wf * m10 - m2) * p.dz);
-        slope[n * 5 + 3] = (float)(m6 * p.dz);
-        slope[n * 5 + 4] = (float)(((double)p.Hf * m10 - m6) * p.dz);
-    }
-    for (int c = tid; c < 32; c += THREADS) {
-        int v = 0;
-        if (c < p.ct) {
-            const int s = c / p.cpw, j = c - s * p.cpw;  // sub-block, cell inside it
-            const int si = s / p.sby, sj = s - si * p.sby;
-            const int jx = j / p.wy, jy = j - jx * p.wy;
-            v = (si * p.wx + jx) | ((sj * p.wy + jy) << 8);
-        }
-        celltab[c] = v;
-    }
-    __syncthreads();  // the only CTA-wide barrier
-
-    // ---- gather role of this lane inside a sub-block
-    const int cg = lane / p.g, gl = lane - cg * p.g;
-    const bool role = cg < p.cpw;
-    constexpr bool kWide = WIDE && V >= 2 && !BWD;
-    const int vstep = kWide ? 1 : p.g;  // distance between the lane's channel vectors
-    const int vec0 = kWide ? (blockIdx.y * p.g + gl) * V : blockIdx.y * (p.g * V) + gl;  // the lane's first vector
-    // channel vectors past the end of the row (ragged last channel block) re-read vector 0, never stored
-    const uint4 *featv[V];
-    float4 *gfv[V];  // backward: where this lane's channel vectors of a texel's gradient live
-    {
-        const size_t cam0 = (size_t)b * p.N * p.Hf * p.Wf * p.vecs;
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            const int vi = (vec0 + v * vstep < p.vecs) ? vec0 + v * vstep : 0;
-            featv[v] = BWD ? nullptr : static_cast<const uint4 *>(p.feat) + cam0 + vi;
-            gfv[v] = BWD ? reinterpret_cast<float4 *>(p.gfeat) + cam0 + vi : nullptr;
-        }
-    }
-    const int my_tab = celltab[lane];
-
-    for (int rep = 0; rep < p.reps; ++rep) {
-        // ---- which super-block: ids run along y inside bands of `band` rows of super-blocks
-        const int id = (blockIdx.x * WARPS + warp) * p.reps + rep;
-        const int per_band = p.band * p.blocks_y;
-        const int bandi = id / per_band, rem = id - bandi * per_band;
-        const int by = rem / p.band, bx = bandi * p.band + (rem - by * p.band);
-        if (bx >= p.blocks_x) continue;  // warp-uniform
-        const int ix0 = bx * (p.sbx * p.wx), iy0 = by * (p.sby * p.wy);
-
-        unsigned in_mask;  // bit c: cell c of the super-block is inside the grid
-        {
-            const int lx = my_tab & 0xff, ly = my_tab >> 8;
-            const bool in = (lane < p.ct) && (ix0 + lx < p.X) && (iy0 + ly < p.Y);
-            const double nan = __longlong_as_double(0x7ff8000000000000LL);
-            sm.cellxy[lane] = make_double2(in ? p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx : nan,
-                                           in ? p.y_min + ((double)(iy0 + ly) + 0.5) * p.dy : nan);
-            sm.cell_count[lane] = 0;
-            in_mask = __ballot_sync(FULL, in);
-        }
-
-        float2 acc[V][PV];
-#pragma unroll
-        for (int v = 0; v < V; ++v)
-#pragma unroll
-            for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
-        unsigned touched = 0;  // bit s: this lane has already stored its part of sub-block s
-
-        // Backward of MEAN_OVER_VALID: the cell's whole count scales every contribution, so count first.
-        if (BWD && p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) {
-            for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
-                const int kc1 = min(p.Z, kc0 + p.zc);
-                if (lane == 0) *sm.n_walkers = 0;
-                __syncwarp();
-                phase_a(p, sm, mats, slope, in_mask, kc0, kc1, lane);
-                __syncwarp();
-                const int n_walkers = min(*sm.n_walkers, p.wcap);
-                for (int wi = lane; wi < n_walkers; wi += 32) {
-                    const uint32_t wd = sm.walkers[wi];
-                    const int c = wd & 0xff, n = (wd >> 8) & 0x3f, k0 = kc0 + ((wd >> 14) & 0x1ff), k1 = k0 + (wd >> 23);
-                    ColumnWalk cw;
-                    cw.init(p, mats, n, sm.cellxy[c]);
-                    int cnt = 0;
-                    for (int k = k0; k <= k1; ++k) {
-                        Sample s;
-                        cnt += cw.sample(k, s) ? 1 : 0;
-                    }
-                    if (cnt) atomicAdd(&sm.cell_count[c], cnt);
-                }
-                __syncwarp();
-            }
-        }
-
-        for (int kc0 = 0; kc0 < p.Z; kc0 += p.zc) {
-            const int kc1 = min(p.Z, kc0 + p.zc);  // chunk [kc0, kc1)
-            if (lane == 0) *sm.n_walkers = 0;
-            if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM)
-                for (int i = lane; i < (p.ct * p.zc + 3) / 4; i += 32) sm.den[i] = 0u;
-            __syncwarp();
-
-            phase_a(p, sm, mats, slope, in_mask, kc0, kc1, lane);
-            __syncwarp();
-            const int n_walkers = min(*sm.n_walkers, p.wcap);
-
-            // ---- Eq. 1 mode: den_z = sum_n M_n for every (cell, z) of the chunk, before any weight
-            if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
-                for (int wi = lane; wi < n_walkers; wi += 32) {
-                    const uint32_t wd = sm.walkers[wi];
-                    const int c = wd & 0xff, n = (wd >> 8) & 0x3f, k0 = kc0 + ((wd >> 14) & 0x1ff), k1 = k0 + (wd >> 23);
-                    ColumnWalk cw;
-                    cw.init(p, mats, n, sm.cellxy[c]);
-                    for (int k = k0; k <= k1; ++k) {
-                        Sample s;
-                        if (cw.sample(k, s)) {
-                            const int di = c * p.zc + (k - kc0);
-                            atomicAdd(&sm.den[di >> 2], 1u << (8 * (di & 3)));
-                        }
-                    }
-                }
-                __syncwarp();
-            }
-
-            // ---- rounds: walk (every lane runs its walkers lane, lane + 32, ... until one has to stop
-            // because its cell's list is full) -> gather all sub-blocks; repeat while walkers are left
-            int resume = lane;
-            bool has_state = false;
-            while (true) {
-                sm.list_count[lane] = 0;
-                sm.list_end[lane] = 0x7fffffff;
-                __syncwarp();
-
-                bool pending = false;
-                for (int wi = resume; wi < n_walkers; wi += 32) {
-                    const uint32_t wd = sm.walkers[wi];
-                    const int wc = wd & 0xff, wn = (wd >> 8) & 0x3f;
-                    const int k0 = kc0 + ((wd >> 14) & 0x1ff), kend = k0 + (int)(wd >> 23);
-                    Walker w;
-                    if (has_state) {
-                        w.k = (int)sm.wsave[0 * 32 + lane];
-                        w.ox = (int)sm.wsave[1 * 32 + lane];
-                        w.oy = (int)sm.wsave[2 * 32 + lane];
-                        w.vcount = (int)sm.wsave[3 * 32 + lane];
-                        w.uL = __uint_as_float(sm.wsave[4 * 32 + lane]);
-                        w.uR = __uint_as_float(sm.wsave[5 * 32 + lane]);
-                        w.lL = __uint_as_float(sm.wsave[6 * 32 + lane]);
-                        w.lR = __uint_as_float(sm.wsave[7 * 32 + lane]);
-                        w.open = sm.wsave[8 * 32 + lane] != 0u;
-                        has_state = false;
-                    } else {
-                        w.k = k0, w.ox = 0, w.oy = 0, w.vcount = 0, w.open = false;
-                        w.uL = w.uR = w.lL = w.lR = 0.f;
-                    }
-                    if (run_walker(p, sm, mats, w, wc, wn, kend, kc0, sm.list + wc * (p.lcap + 1))) {
-                        if (w.vcount && !(BWD && p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID))
-                            atomicAdd(&sm.cell_count[wc], w.vcount);
-                    } else {
-                        sm.wsave[0 * 32 + lane] = (uint32_t)w.k;
-                        sm.wsave[1 * 32 + lane] = (uint32_t)w.ox;
-                        sm.wsave[2 * 32 + lane] = (uint32_t)w.oy;
-                        sm.wsave[3 * 32 + lane] = (uint32_t)w.vcount;
-                        sm.wsave[4 * 32 + lane] = __float_as_uint(w.uL);
-                        sm.wsave[5 * 32 + lane] = __float_as_uint(w.uR);
-                        sm.wsave[6 * 32 + lane] = __float_as_uint(w.lL);
-                        sm.wsave[7 * 32 + lane] = __float_as_uint(w.lR);
-                        sm.wsave[8 * 32 + lane] = w.open ? 1u : 0u;
-                        has_state = true;
-                        pending = true;
-                        resume = wi;
-                        break;
-                    }
-                }
-                if (!pending) resume = n_walkers;
-                __syncwarp();
-                const bool more = __any_sync(FULL, pending);
-                const bool final = !more && kc1 >= p.Z;  // last commit of this super-block
-
-                // ---- gather, one sub-block at a time
-                for (int s = 0; s < p.sbn; ++s) {
-                    const int cell = s * p.cpw + (role ? cg : 0);
-                    const bool lane_on = role && ((in_mask >> cell) & 1u);
-                    const int nrec = lane_on ? min(sm.list_count[cell], sm.list_end[cell]) : 0;
-                    const int maxn = __reduce_max_sync(FULL, nrec);
-                    if (BWD) {
-                        if (nrec > 0) {
-                            const int tab = celltab[cell];
-                            const size_t ocell = ((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8));
-                            const int count = sm.cell_count[cell];
-                            const float gscale = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID)
-                                                     ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-                            float4 go[V];
-                            bool on[V];
-#pragma unroll
-                            for (int v = 0; v < V; ++v) {
-                                const int vi = vec0 + v * vstep;
-                                go[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                on[v] = vi < p.vecs;
-                                if (on[v]) {
-                                    go[v] = __ldg(reinterpret_cast<const float4 *>(p.gout + ocell * p.C) + vi);
-                                    go[v].x *= gscale, go[v].y *= gscale, go[v].z *= gscale, go[v].w *= gscale;
-                                }
-                            }
-                            scatter_list<V>(go, on, sm.list + cell * (p.lcap + 1), nrec, gfv);
-                        }
-                        continue;
-                    }
-                    if (p.sbn > 1) {
-#pragma unroll
-                        for (int v = 0; v < V; ++v)
-#pragma unroll
-                            for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
-                    }
-                    gather_list<V, BF16, kWide>(acc, sm.list + cell * (p.lcap + 1), nrec, maxn, featv);
-                    const bool stored = (touched >> s) & 1u;
-                    // one sub-block per warp: accumulators live on; several: add to the stored partial sums
-                    const bool write = lane_on && (p.sbn > 1 ? (nrec > 0 || (final && (!stored ||
-                                                   p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID))) : final);
-                    if (write) {
-                        const int count = sm.cell_count[cell];
-                        const float g = (final && p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID)
-                                            ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-                        const int tab = celltab[cell];
-                        const size_t ocell = ((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8));
-                        float *o = p.out + ocell * p.C;
-#pragma unroll
-                        for (int v = 0; v < V; ++v) {
-                            const int vi = vec0 + v * vstep;
-                            if (vi < p.vecs) {
-#pragma unroll
-                                for (int e = 0; e < PV; e += 2) {
-                                    float4 *dst = reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2);
-                                    float4 val = make_float4(acc[v][e].x, acc[v][e].y, acc[v][e + 1].x, acc[v][e + 1].y);
-                                    if (stored) {
-                                        const float4 prev = *dst;
-                                        val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
-                                    }
-                                    val.x *= g, val.y *= g, val.z *= g, val.w *= g;
-                                    if (p.accumulate) {  // one sub-block per warp: `dst` still holds the other levels' sum
-                                        const float4 prev = *dst;
-                                        val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
-                                    }
-                                    if (p.out_bf16) {  // only with one sub-block per warp: this is the single, final store
-                                        uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C;
-                                        *reinterpret_cast<uint2 *>(ob + (size_t)vi * (PV * 2) + e * 2) =
-                                            make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
-                                    } else if (final) {
-                                        __stcs(dst, val);
-                                    } else {
-                                        *dst = val;
-                                    }
-                                }
-                            }
-                        }
-                        touched |= 1u << s;
-                    }
-                    if (final && lane_on && p.count_out && gl == 0 && blockIdx.y == 0) {
-                        const int tab = celltab[cell];
-                        p.count_out[((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8))] = sm.cell_count[cell];
-                    }
-                }
-                __syncwarp();
-                if (!more) break;
-            }
-        }
-        __syncwarp();
-    }
-}
+// Kernel 2: tiled (forward and backward), see vt_tiled.cuh
+#include "vt_tiled.cuh"
 
 // ------------------------------------------------------------------------------------------
 // Kernel 3: FlashSCA -- spatial cross-attention with on-the-fly projection (paper Sec. 4.4).  One warp per
@@ -1308,6 +681,8 @@ bool tiled_applicable(const flashbev_vt_params *p)
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
     if (((size_t)p->C * elem) % 16) return false;
     if (((uintptr_t)p->features % 16) || ((uintptr_t)p->out % 16)) return false;
+    if (p->Z > 32767) return false;  // a column's interval of height bins is kept in two 16-bit fields
+    if (p->reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM && p->Z > 16384) return false;  // per-height camera counts on chip
     const double vecs_total = (double)p->N * p->feat_h * p->feat_w * (double)((size_t)p->C * elem / 16);
     return vecs_total < 2147483648.0;
 }
@@ -1337,86 +712,54 @@ cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t sm
     }
 }
 
-// Chooses the channel mapping, super-block shape, chunking and grid of the tiled kernel.
+// Chooses the channel mapping, sub-block shape, list size and grid of the tiled kernel.
 flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V, int &warps, dim3 &grid, size_t &smem,
                                 bool accumulate = false)
 {
     k = base_params(p, accumulate);
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     const int elem = bf16 ? 2 : 4;
+    const bool eq1 = p->reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM;
     k.vecs = p->C * elem / 16;
+    k.rstep = p->feat_w > 1 ? k.vecs : 0;
+    k.nvec_cam = p->N * p->feat_h * p->feat_w * k.vecs;  // < 2^31: tiled_applicable
 
     // channel mapping: V vectors per lane, g lanes per cell
     V = p->tune[0];
     int g = p->tune[1];
     if (!(V == 1 || V == 2 || V == 4) || g < 1 || g > 32) V = 0, g = 0;
     if (!V) {
-        // tall columns: the geometry of a column dominates, eight cells per sub-block amortise it better
+        // tall columns: eight cells per warp amortise the per-warp geometry better
         if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
         else if (k.vecs <= 8) V = 1, g = k.vecs;
         else if (k.vecs <= 16) V = (k.vecs % 2 == 0) ? 2 : 1, g = (k.vecs + V - 1) / V;
-        else if (k.vecs < 24 || (k.vecs <= 32 && p->Z >= 16)) V = 2, g = (k.vecs + 1) / 2;  // (16+ bins: 0-17 % over V = 4)
+        else if (k.vecs < 24 || (k.vecs <= 32 && p->Z >= 16)) V = 2, g = (k.vecs + 1) / 2;
         else V = 4, g = (k.vecs + 3) / 4;  // wide texels: four vectors per lane keep 2-5 cells in a sub-block
         if (g > 32) g = 32;
     }
     warps = p->tune[3] & 0xf;
     if (!(warps == 1 || warps == 2 || warps == 4 || warps == 8)) warps = 4;
     k.g = g;
-    k.cpw = 32 / g;
-    if (k.cpw > 8) k.cpw = 8;
+    int cpw = std::min(32 / g, kMaxCells);
+    cpw = std::min(cpw, std::max(1, 64 / p->N));            // column descriptors per warp: cells * cameras <= 64
+    if (eq1) cpw = std::min(cpw, std::max(1, 16384 / p->Z));  // per-(cell, height) camera counts: <= 16 KB per warp
     // sub-block of wx x wy cells, near-square, y (the contiguous output axis) the longer side
-    k.wy = (k.cpw % 2 == 0) ? 2 : (k.cpw == 3 ? 3 : 1);
-    if (k.cpw == 8) k.wy = 4;
-    if (k.cpw == 6) k.wy = 3;
-    if (k.cpw == 5 || k.cpw == 7) k.wy = k.cpw;
-    k.wx = k.cpw / k.wy;
+    k.wy = (cpw % 2 == 0) ? 2 : (cpw == 3 ? 3 : 1);
+    if (cpw == 8) k.wy = 4;
+    if (cpw == 6) k.wy = 3;
+    if (cpw == 5 || cpw == 7) k.wy = cpw;
+    k.wx = cpw / k.wy;
     k.cpw = k.wx * k.wy;
-    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 64) ? p->tune[2] : (p->Z < 16 ? 4 : (p->Z <= 32 ? 8 : 16));
-    const int runs = (p->Z + k.walk - 1) / k.walk;  // walkers per column when all of Z is one chunk
-
-    // super-block: as many sub-blocks as keep the whole height range in one chunk (<= 8 cells: larger
-    // ones pack the geometry lanes better but leave too few warps to overlap geometry with gathers)
-    // record slots per warp: 16 and more height bins write long lists, and every list that fills up costs another
-    // walk-and-gather round (measured: 64 bins, 8 cells: 128 slots 458 us, 384 slots 368 us, 512 slots 399 us;
-    // 16 bins, 8 cells: 192 slots 172 us, 384 slots 162 us, 512 slots 173 us -- shared memory then costs warps)
-    const int slot_budget = p->Z >= 16 ? 384 : 192;
-    int sbx = (p->tune[3] >> 4) & 0xf, sby = (p->tune[3] >> 8) & 0xf;
-    if (k.out_bf16 || k.accumulate) {
-        // a rounded output cannot take partial sums, and an output that already holds another level's result
-        // must be added once, at the end: keep the accumulators in registers
-        sbx = sby = 1;
-    } else if (sbx < 1 || sby < 1 || sbx * sby * k.cpw > 32) {
-        sbx = sby = 1;
-        while (true) {
-            const bool grow_x = sby > sbx;  // first along y, the contiguous output axis (1-2 % on three of four shapes)
-            const int nx = grow_x ? sbx * 2 : sbx, ny = grow_x ? sby : sby * 2;
-            const int ct = nx * ny * k.cpw;
-            // keep the whole height range in one chunk and leave each cell a list of ~1.5 Z + 4 records
-            if (ct > 8 || (long long)ct * p->N * runs > 512 || ct * (3 * p->Z / 2 + 4) > slot_budget) break;
-            // small problems: rather one warp per sub-block than idle SMs (a warp's latency is the kernel's)
-            if ((long long)p->B * p->X * p->Y / ct < (long long)sm_count() * 24) break;
-            sbx = nx, sby = ny;
-        }
-    }
-    k.sbx = sbx, k.sby = sby, k.sbn = sbx * sby;
-    k.ct = k.sbn * k.cpw;
-    k.ct_inv = (65536 + k.ct - 1) / k.ct;
-    k.blocks_x = (p->X + sbx * k.wx - 1) / (sbx * k.wx);
-    k.blocks_y = (p->Y + sby * k.wy - 1) / (sby * k.wy);
+    k.blocks_x = (p->X + k.wx - 1) / k.wx;
+    k.blocks_y = (p->Y + k.wy - 1) / k.wy;
     k.band = 4;
     k.reps = (p->tune[3] >> 12) & 0xf;
     if (k.reps < 1) k.reps = 1;
-    k.slots = p->Z >= 16 ? slot_budget : (k.sbn > 1 ? 192 : 128);
-    k.lcap = k.slots / k.ct;
-    // height chunk: all walkers of a chunk must fit the warp's descriptor array
-    k.wcap = (int)std::min<long long>(512, std::max<long long>(128, (long long)k.ct * p->N * runs));
-    if (k.wcap < k.ct * p->N) k.wcap = k.ct * p->N;
-    const int per_column = k.wcap / (k.ct * p->N);
-    int zc = per_column * k.walk;
-    if (zc > 256) zc = 256;
-    if (zc >= p->Z) zc = p->Z;
-    else if (zc >= 4) zc = (zc / 4) * 4;
-    k.zc = zc;
+    // record slots per warp: about the records of a typical sub-block, so that most lists take one round
+    if (p->tune[2] >= 64) k.slots = std::min(p->tune[2], 2048);
+    else k.slots = std::min(384, std::max(96, (k.cpw * (std::min(p->Z, 64) + 16) + 31) / 32 * 32));
+    k.ncap = k.cpw * p->N;
+    k.den_bytes = eq1 ? (int)align16((size_t)k.cpw * p->Z) : 0;
 
     const long long bands = (k.blocks_x + k.band - 1) / k.band;
     const long long ids = bands * k.band * k.blocks_y;
@@ -1428,8 +771,8 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     // texels per cell where the strided 16-byte segments of a cell would not cover whole 128-byte lines
     k.wide = warps == 4 && (V == 2 || (V == 4 && (p->tune[3] & 0x20000))) && k.vecs % V == 0 && (uintptr_t)p->features % 32 == 0 &&
              (bf16 || (g * 16) % 128 != 0 || (p->tune[3] & 0x20000)) && !(p->tune[3] & 0x10000);
-    smem = align16(cta_table_bytes(p->N)) +
-                        (size_t)warps * warp_smem_layout(nullptr, nullptr, k.ct, k.slots, k.zc, k.wcap);
+    smem = cta_table_bytes(p->N) + (size_t)warps * warp_smem_layout(nullptr, nullptr, k.slots, k.ncap, k.den_bytes);
+    if (smem > 200 * 1024) return FLASHBEV_UNSUPPORTED;
     return FLASHBEV_OK;
 }
 

@@ -47,16 +47,22 @@ struct KParams {
     // tiled kernel only
     int vecs;                   // 16-byte vectors per texel (C * elem / 16)
     int g;                      // lanes per cell
-    int cpw;                    // cells per sub-block (= wx * wy <= 8): the cells one warp works on at a time
+    int cpw;                    // cells per sub-block (= wx * wy <= 8): the cells one gather pass covers
     int wx, wy;                 // sub-block size in cells (x, y)
-    int blocks_x, blocks_y;     // sub-blocks per batch element
-    int band, reps;             // sub-block order: bands of `band` rows; sub-blocks per warp
-    int slots;                  // record slots per warp (>= 64)
-    int ncap;                   // column descriptors per warp (= cpw * N)
+    int sbx, sby, sbn;          // sub-blocks per super-block (x, y, total)
+    int ct;                     // cells per super-block (<= 32)
+    float inv_n;                // 1 / N
+    int blocks_x, blocks_y;     // super-blocks per batch element
+    int band, reps;             // super-block order: bands of `band` rows; super-blocks per warp
+    int walk;                   // height bins per run (2 walk <= slots)
+    int slots;                  // record slots per warp
+    int colcap;                 // column descriptors per warp (>= cpw * N)
+    int wcap;                   // runs per warp (= column descriptors per warp * ceil(Z / walk))
     int den_bytes;              // bytes of the per-(cell, height) camera counts per warp (Eq. 1 mode, else 0)
     int rstep;                  // distance (16-byte vectors) from a record's first tap to its second: vecs, or 0 on 1-texel-wide maps
     int nvec_cam;               // N * Hf * Wf * vecs: vectors of one batch element's feature maps (bounds-checked build)
     int wide;                   // host side: use the instance with adjacent channel vectors and 256-bit loads
+    int dbg;
     unsigned *err;              // bounds-checked build: device word that counts out-of-range indices (may be null)
 };
 
@@ -712,7 +718,7 @@ cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t sm
     }
 }
 
-// Chooses the channel mapping, sub-block shape, list size and grid of the tiled kernel.
+// Chooses the channel mapping, super-block shape, run length, list size and grid of the tiled kernel.
 flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V, int &warps, dim3 &grid, size_t &smem,
                                 bool accumulate = false)
 {
@@ -723,13 +729,15 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     k.vecs = p->C * elem / 16;
     k.rstep = p->feat_w > 1 ? k.vecs : 0;
     k.nvec_cam = p->N * p->feat_h * p->feat_w * k.vecs;  // < 2^31: tiled_applicable
+    k.inv_n = 1.0f / (float)p->N;
+    k.dbg = (p->tune[3] >> 28) & 7;
 
     // channel mapping: V vectors per lane, g lanes per cell
     V = p->tune[0];
     int g = p->tune[1];
     if (!(V == 1 || V == 2 || V == 4) || g < 1 || g > 32) V = 0, g = 0;
     if (!V) {
-        // tall columns: eight cells per warp amortise the per-warp geometry better
+        // tall columns: eight cells per sub-block
         if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
         else if (k.vecs <= 8) V = 1, g = k.vecs;
         else if (k.vecs <= 16) V = (k.vecs % 2 == 0) ? 2 : 1, g = (k.vecs + V - 1) / V;
@@ -740,9 +748,8 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     warps = p->tune[3] & 0xf;
     if (!(warps == 1 || warps == 2 || warps == 4 || warps == 8)) warps = 4;
     k.g = g;
-    int cpw = std::min(32 / g, kMaxCells);
-    cpw = std::min(cpw, std::max(1, 64 / p->N));            // column descriptors per warp: cells * cameras <= 64
-    if (eq1) cpw = std::min(cpw, std::max(1, 16384 / p->Z));  // per-(cell, height) camera counts: <= 16 KB per warp
+    int cpw = std::min(32 / g, kMaxCpw);
+    cpw = std::min(cpw, std::max(1, kColCapMax / p->N));  // a sub-block's candidate columns fit the descriptor table
     // sub-block of wx x wy cells, near-square, y (the contiguous output axis) the longer side
     k.wy = (cpw % 2 == 0) ? 2 : (cpw == 3 ? 3 : 1);
     if (cpw == 8) k.wy = 4;
@@ -750,16 +757,52 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     if (cpw == 5 || cpw == 7) k.wy = cpw;
     k.wx = cpw / k.wy;
     k.cpw = k.wx * k.wy;
-    k.blocks_x = (p->X + k.wx - 1) / k.wx;
-    k.blocks_y = (p->Y + k.wy - 1) / k.wy;
+
+    // record slots per warp and bins per run (a run writes at most two records per bin)
+    const int slots_tune = (p->tune[3] >> 20) & 0xff;
+    k.slots = slots_tune ? std::max(64, slots_tune * 16) : 320;
+    // a run is at most `walk` height bins, or `walk` texel rows of a column that moves at most two rows per bin
+    const int units = std::max(p->Z, std::min(p->feat_h, 2 * p->Z + 2));  // per column at most
+    k.walk = (p->tune[2] >= 1 && p->tune[2] <= 256) ? p->tune[2] : 16;
+    k.walk = std::min(k.walk, std::min(units, (k.slots - 2) / 2));
+    k.colcap = std::max(32, (k.cpw * p->N + 7) / 8 * 8);
+    int runs = (units + k.walk - 1) / k.walk;
+    while (k.colcap * runs > 2048 && k.walk < std::min(256, (k.slots - 2) / 2)) {  // keep the run table small: longer runs
+        k.walk = std::min(std::min(256, (k.slots - 2) / 2), k.walk * 2);
+        runs = (units + k.walk - 1) / k.walk;
+    }
+
+    // super-block: about as many cells as fill the record slots in one round (a cell writes roughly 0.7 Z + 8
+    // records on surround rigs), so that the walkers of a round keep most lanes busy
+    int sbx = (p->tune[3] >> 4) & 0xf, sby = (p->tune[3] >> 8) & 0xf;
+    auto fits = [&](int nx, int ny) {
+        const int ct = nx * ny * k.cpw;
+        if (ct > kMaxCt || ct * p->N > 512) return false;
+        if (eq1 && (long long)ct * p->Z > 16384) return false;
+        return true;
+    };
+    if (sbx < 1 || sby < 1 || !fits(sbx, sby)) {
+        static const int shapes[][2] = {{1, 1}, {1, 2}, {2, 2}, {2, 3}, {2, 4}, {3, 3}, {3, 4}, {4, 4}};
+        const int want = std::max(k.cpw, (int)(k.slots / (0.7 * std::min(p->Z, 2 * p->feat_h) + 8.0)));
+        sbx = sby = 1;
+        for (const auto &sh : shapes) {
+            const int ct = sh[0] * sh[1] * k.cpw;
+            if (!fits(sh[0], sh[1]) || ct > want) break;
+            // small problems: rather more warps than idle SMs (a warp's latency is the kernel's)
+            if (ct > k.cpw && (long long)p->B * p->X * p->Y / ct < (long long)sm_count() * 24) break;
+            sbx = sh[0], sby = sh[1];
+        }
+    }
+    if (!fits(sbx, sby)) return FLASHBEV_UNSUPPORTED;
+    k.sbx = sbx, k.sby = sby, k.sbn = sbx * sby;
+    k.ct = k.sbn * k.cpw;
+    k.blocks_x = (p->X + sbx * k.wx - 1) / (sbx * k.wx);
+    k.blocks_y = (p->Y + sby * k.wy - 1) / (sby * k.wy);
     k.band = 4;
     k.reps = (p->tune[3] >> 12) & 0xf;
     if (k.reps < 1) k.reps = 1;
-    // record slots per warp: about the records of a typical sub-block, so that most lists take one round
-    if (p->tune[2] >= 64) k.slots = std::min(p->tune[2], 2048);
-    else k.slots = std::min(384, std::max(96, (k.cpw * (std::min(p->Z, 64) + 16) + 31) / 32 * 32));
-    k.ncap = k.cpw * p->N;
-    k.den_bytes = eq1 ? (int)align16((size_t)k.cpw * p->Z) : 0;
+    k.wcap = k.colcap * runs;
+    k.den_bytes = eq1 ? (int)align16((size_t)k.ct * p->Z) : 0;
 
     const long long bands = (k.blocks_x + k.band - 1) / k.band;
     const long long ids = bands * k.band * k.blocks_y;
@@ -771,7 +814,8 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     // texels per cell where the strided 16-byte segments of a cell would not cover whole 128-byte lines
     k.wide = warps == 4 && (V == 2 || (V == 4 && (p->tune[3] & 0x20000))) && k.vecs % V == 0 && (uintptr_t)p->features % 32 == 0 &&
              (bf16 || (g * 16) % 128 != 0 || (p->tune[3] & 0x20000)) && !(p->tune[3] & 0x10000);
-    smem = cta_table_bytes(p->N) + (size_t)warps * warp_smem_layout(nullptr, nullptr, k.slots, k.ncap, k.den_bytes);
+    smem = align16(cta_table_bytes(p->N)) +
+           (size_t)warps * warp_smem_layout(nullptr, nullptr, k.slots, k.colcap, k.wcap, k.ct, k.ct * p->N, k.den_bytes);
     if (smem > 200 * 1024) return FLASHBEV_UNSUPPORTED;
     return FLASHBEV_OK;
 }

@@ -1,30 +1,31 @@
 // Tiled Sampling-VT kernel (forward and backward) for B200 (sm_100a).  Included by flashbev.cu inside its
-// anonymous namespace, after the shared helpers (KParams, fast_rcp, kDepthMin, FB_IDX).
+// anonymous namespace, after the shared helpers (KParams, fast_rcp, kDepthMin, FB_IDX, pack_bf16x2).
 //
-// A WARP owns a sub-block of up to 8 adjacent BEV cells and works through it alone (__syncwarp only; the CTA
-// shares nothing but the per-batch-element camera tables staged once at kernel start).  Everything that does
-// not depend on the channel is computed once per (cell, camera, height) and turned into a compact list of
-// "row records" in shared memory before a single feature is read (paper Sec. 3.3: the projection, validity
-// test and bilinear weights of Algorithm 2, hoisted out of the channel dimension):
+// A WARP owns a super-block of up to 32 adjacent BEV cells (sbn sub-blocks of cpw <= 8 cells) and works through
+// it alone (__syncwarp only; the CTA shares nothing but the per-batch-element tables staged once at kernel
+// start).  Everything that does not depend on the channel is computed once per (cell, camera, height) and
+// turned into a compact list of "row records" in shared memory before a single feature is read (paper Sec. 3.3:
+// the projection, validity test and bilinear weights of Algorithm 2, hoisted out of the channel dimension):
 //
-//   1. columns   one lane per (cell, camera): the five validity conditions are linear in the height once the
-//                depth is positive, so the valid height bins of a column form one interval [klo, khi]; it is
-//                found in closed form (float, conservative) and its two ends are confirmed with the exact
-//                fp64 test.  The surviving columns are compacted (ballot) into column descriptors.  The cell's
-//                valid-sample count and the per-height camera counts of Eq. 1 follow from the intervals alone.
-//   2. items     the columns' work is cut into items that the 32 lanes take in order, one item per lane:
-//                - a camera without pitch or roll sees a column under one texel column (x0, tx constant) with
-//                  fy affine in the bin index; if several bins share a texel row the item is a texel ROW: the
-//                  bins that fall into it and their summed weights are arithmetic series (closed form);
-//                - otherwise the item is a height BIN; the lane that starts a run of bins on the same texel
-//                  rows sums the run (and the lower-row weights of the run just before it, when that run ends
-//                  one row above), so successive bins that touch the same row still give one record.
-//                Records {left tap, right tap, wL, wR} are written in item order at positions given by a
-//                ballot/popc prefix: no atomics, the list of every cell is contiguous and its order fixed.
-//   3. gather    g lanes per cell, V 16-byte channel vectors per lane: per record two 128- or 256-bit loads per
-//                vector and packed fp32 FMAs into register accumulators.  A list that does not fit its slots is
-//                consumed in several rounds; the accumulators stay in registers, so every output vector is
-//                written exactly once, with a streaming store.
+//   1a. candidates  one lane per (cell, camera): the five validity conditions are linear in the height once the
+//                   depth is positive, so a column whose two end bins both fail the same condition (widened by a
+//                   texel) has no valid bin.  About 4/5 of the candidates end here; the rest are compacted.
+//   1b. columns     one lane per surviving column: the valid bins form ONE interval; it comes in closed form
+//                   (float, conservative) and its two ends are confirmed with the exact fp64 test.  A camera
+//                   without pitch or roll sees the column under one texel column (x0, tx constant) with fy affine
+//                   in the bin index: then the texel rows the column touches, and so the number of records it
+//                   will write, follow in closed form.  Columns are cut into runs of at most `walk` bins; a
+//                   prefix sum over the record counts gives every run its place in the list, so the records of a
+//                   cell are contiguous, their order is fixed and no atomics are needed.  The valid-sample count
+//                   of a cell and the per-height camera counts of Eq. 1 follow from the intervals alone.
+//   2.  walkers     one lane per run: successive bins that land on the same texel rows are merged into one
+//                   record {left tap, right tap, wL, wR} per row.  Affine columns cost one fp64 FMA and a floor
+//                   per bin; the others are projected bin by bin in fp64 (their records are counted by a first
+//                   sweep of the same walker).
+//   3.  gather      one sub-block at a time: g lanes per cell, V 16-byte channel vectors per lane; per record two
+//                   128- or 256-bit loads per vector and packed fp32 FMAs into register accumulators.  Runs that
+//                   do not fit the record slots are taken in several rounds; the accumulators of the sub-block
+//                   stay in registers, so every output vector is written exactly once, with a streaming store.
 // The backward instance replaces step 3 by the transpose: fp32 vector reductions of w * grad_out into the
 // feature gradient.
 //
@@ -32,36 +33,54 @@
 //   CTA  : double mats[N][12]   rows 0..2 of lidar2img[b][n], rows 0/1 pre-scaled to feature texels
 //          float  slope[N][5]   d/dk of the five validity conditions
 //          int    camfast[N]    1: the camera's depth and horizontal texel coordinate do not depend on height
-//   warp : int4    rec[slots]    row records of the current round
-//          ColDesc col[ncap]     descriptors of the valid columns (ncap = cells * N)
-//          double2 cellxy[8]     voxel-centre (x_w, y_w) of the cells (NaN: outside the grid)
-//          int     cfirst[9], cstart[8], cend[8], cnt[8]
-//          uint8   den[cells * Z]   cameras per (cell, height bin), Eq. 1 mode only
+//          int    celltab[32]   position of cell c inside a super-block: lx | ly << 8
+//   warp : int     roff[slots + 4] row records of the current round: vector index of the first tap (the second follows
+//          float2  rw[slots + 4]   `rstep` vectors later) and the two weights (+ slack that is read, never used)
+//          ColDesc col[ccap]       columns of the current segment, (cell, camera) order
+//          uint32  wk[wcap]        runs: column | first bin << 8 | (bins - 1) << 24
+//          int     woff[wcap + 1]  records before run w
+//          int     colw[ccap + 1]  runs before column j
+//          uint16  cand[ct * N]    surviving candidates: cell | camera << 8
+//          double2 cellxy[32], int cfirst[33], int cnt[32]
+//          uint8   den[ct * Z]     cameras per (cell, height bin), Eq. 1 mode only
 
-constexpr int kMaxCells = 8;        // cells per warp
-constexpr int kKindRows = 0;        // item = texel row of a height-independent column (closed form)
-constexpr int kKindBinsFast = 1;    // item = height bin, height-independent column
-constexpr int kKindBinsGeneral = 2; // item = height bin, full projection per bin
+#ifndef FB_EMIT_INLINE
+#define FB_EMIT_INLINE __forceinline__
+#endif
+#ifndef FB_U_BF16V2
+#define FB_U_BF16V2 3
+#endif
+#ifndef FB_WARPS_PER_SM
+#define FB_WARPS_PER_SM 20
+#endif
+
+constexpr int kMaxCt = 32;   // cells per super-block
+constexpr int kMaxCpw = 8;   // cells per sub-block
+constexpr int kColCapMax = 64;  // column descriptors per warp (a sub-block never has more candidates than that)
+constexpr int kWalkIlp = 1;  // height bins whose geometry a general walker evaluates independently
 
 struct __align__(16) ColDesc {
-    double a, s;     // fast: fy(k') = a + k' s, rows ascending with k' (s >= 0); general: a0, a1 (rows 0/1 at z = 0)
-    double inv;      // rows: ~1 / s; general: a2 (row 2 at z = 0)
-    int offc;        // fast: vector index of the left loadable texel of the column at row 0
-    int r0;          // fast: floor(a)
-    float cl, cr;    // fast: horizontal weights of the two loadable texels (an out-of-map tap is folded to weight 0)
-    int istart;      // first item of the column in the warp's item order
-    int nitems;
-    int kk;          // klo | khi << 16
-    int meta;        // cell | camera << 8 | kind << 16 | reversed << 18 | first column of cell << 19 | last << 20
-    int pad0, pad1;
+    double d0, d1;  // affine: fy(k') = d0 + k' d1 with d1 >= 0 (bins renumbered so that rows ascend); general: a0, a1
+    union {
+        double d2;  // general: a2  (a_i = row i of the scaled matrix applied to (x_w, y_w, 0, 1))
+        struct {
+            int offc;   // affine: vector index of the column's first loaded texel at row 0
+            float tx;   // affine: horizontal fraction
+        } f;
+    };
+    int kk;    // klo | khi << 16: the valid bins
+    int meta;  // cell | camera << 6 | affine << 12 | reversed << 13 | edge << 14 (0 interior, 1 left tap outside, 2 right tap outside)
 };
-static_assert(sizeof(ColDesc) == 64, "column descriptor is four 16-byte words");
+static_assert(sizeof(ColDesc) == 32, "column descriptor is two 16-byte words");
 
 struct WarpSmem {
-    int4 *rec;
+    int *roff;
+    float2 *rw;
     ColDesc *col;
+    uint32_t *wk;
+    int *woff, *colw, *cfirst, *cnt;
+    uint16_t *cand;
     double2 *cellxy;
-    int *cfirst, *cstart, *cend, *cnt;
     unsigned char *den;
 };
 
@@ -69,10 +88,12 @@ __host__ __device__ inline size_t align16(size_t v) { return (v + 15) & ~(size_t
 
 __host__ __device__ inline size_t cta_table_bytes(int N)
 {
-    return align16((size_t)N * 12 * sizeof(double)) + align16((size_t)N * 5 * sizeof(float)) + align16((size_t)N * sizeof(int));
+    return align16((size_t)N * 12 * sizeof(double)) + align16((size_t)N * 5 * sizeof(float)) + align16((size_t)N * sizeof(int)) +
+           kMaxCt * sizeof(int);
 }
 
-__host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem *t, int slots, int ncap, int den_bytes)
+__host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem *t, int slots, int colcap, int wcap, int ct, int ncand,
+                                                   int den_bytes)
 {
     size_t o = 0;
     auto take = [&](size_t bytes) {
@@ -80,31 +101,34 @@ __host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem
         o += align16(bytes);
         return ptr;
     };
-    unsigned char *p0 = take((size_t)slots * sizeof(int4));
-    unsigned char *p1 = take((size_t)ncap * sizeof(ColDesc));
-    unsigned char *p2 = take((size_t)kMaxCells * sizeof(double2));
-    unsigned char *p3 = take((size_t)(4 * kMaxCells + 4) * sizeof(int));
-    unsigned char *p4 = take((size_t)den_bytes);
+    unsigned char *p0 = take((size_t)(slots + 4) * sizeof(float2));
+    unsigned char *p0b = take((size_t)(slots + 4) * sizeof(int));
+    unsigned char *p1 = take((size_t)colcap * sizeof(ColDesc));
+    unsigned char *p2 = take((size_t)ct * sizeof(double2));
+    unsigned char *p3 = take((size_t)wcap * sizeof(uint32_t));
+    unsigned char *p4 = take((size_t)(wcap + 1) * sizeof(int));
+    unsigned char *p5 = take((size_t)(colcap + 1) * sizeof(int));
+    unsigned char *p6 = take((size_t)(2 * kMaxCt + 1) * sizeof(int));
+    unsigned char *p7 = take((size_t)ncand * sizeof(uint16_t));
+    unsigned char *p8 = take((size_t)den_bytes);
     if (t) {
-        t->rec = reinterpret_cast<int4 *>(p0);
+        t->rw = reinterpret_cast<float2 *>(p0);
+        t->roff = reinterpret_cast<int *>(p0b);
         t->col = reinterpret_cast<ColDesc *>(p1);
         t->cellxy = reinterpret_cast<double2 *>(p2);
-        t->cfirst = reinterpret_cast<int *>(p3);
-        t->cstart = t->cfirst + kMaxCells + 1;
-        t->cend = t->cstart + kMaxCells;
-        t->cnt = t->cend + kMaxCells;
-        t->den = p4;
+        t->wk = reinterpret_cast<uint32_t *>(p3);
+        t->woff = reinterpret_cast<int *>(p4);
+        t->colw = reinterpret_cast<int *>(p5);
+        t->cfirst = reinterpret_cast<int *>(p6);
+        t->cnt = t->cfirst + kMaxCt + 1;
+        t->cand = reinterpret_cast<uint16_t *>(p7);
+        t->den = p8;
     }
     return o;
 }
 
-// One height bin of a column: bilinear corner (x0, y0), vertical fraction, and the horizontal weights of the
-// two texels that are actually loaded (xc, xc + 1 with xc inside the map; an out-of-map tap weighs 0).
-struct Tap {
-    int x0, y0, xc;
-    float cl, cr, ty;
-};
-
+// Horizontal weights of the two texels a record loads (xc, xc + 1, both inside the map): an out-of-map tap
+// weighs 0 and the in-map one takes the slot that keeps both addresses loadable.
 __device__ __forceinline__ void fold_x(int x0, float tx, int Wf, int &xc, float &cl, float &cr)
 {
     if (x0 < 0) {                 // left tap outside: the right tap is texel 0, loaded as the record's first tap
@@ -143,42 +167,41 @@ __device__ __forceinline__ void ldg_pair(const uint4 *ptr, uint4 &a, uint4 &b)
 }
 
 // Gather of one cell list by its channel lanes, U records per iteration.  Every record is two taps of one
-// texel row, both always loadable.  Lanes whose list is shorter than the warp's longest repeat their last
-// record with weight 0; lanes with no records do nothing.
+// texel row, both always loadable.  The slots after a list hold loadable offsets too (another cell's records,
+// older ones, or zeros): the last iteration reads them and gives them weight 0.
 template <int V, bool BF16, bool WIDE>
-__device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int4 *list, int nrec, int maxn,
+__device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int *loff, const float2 *lw, int nrec, int rstep,
                                             const uint4 *const (&featv)[V])
 {
-    constexpr int U = V == 1 ? 4 : (V == 2 ? (BF16 ? 3 : 2) : 1);
-    if (nrec <= 0) return;
-    const int last = nrec - 1;
-    for (int j = 0; j < maxn; j += U) {
-        int4 r[U];
+    constexpr int U = V == 1 ? 4 : (V == 2 ? (BF16 ? FB_U_BF16V2 : 2) : 1);
+    for (int j = 0; j < nrec; j += U) {
+        int ro[U];
+        float2 rw[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) r[u] = list[min(j + u, last)];
+        for (int u = 0; u < U; ++u) ro[u] = loff[j + u], rw[u] = lw[j + u];
         uint4 t[U][2][V];
         if (WIDE) {  // the lane's vectors are adjacent: V / 2 loads of 32 bytes per tap
 #pragma unroll
             for (int u = 0; u < U; ++u)
 #pragma unroll
                 for (int v = 0; v + 1 < V; v += 2) {
-                    ldg_pair(featv[v] + r[u].x, t[u][0][v], t[u][0][v + 1]);
-                    ldg_pair(featv[v] + r[u].y, t[u][1][v], t[u][1][v + 1]);
+                    ldg_pair(featv[v] + ro[u], t[u][0][v], t[u][0][v + 1]);
+                    ldg_pair(featv[v] + ro[u] + rstep, t[u][1][v], t[u][1][v + 1]);
                 }
         } else {
 #pragma unroll
             for (int u = 0; u < U; ++u)
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
-                    t[u][0][v] = __ldg(featv[v] + r[u].x);
-                    t[u][1][v] = __ldg(featv[v] + r[u].y);
+                    t[u][0][v] = __ldg(featv[v] + ro[u]);
+                    t[u][1][v] = __ldg(featv[v] + ro[u] + rstep);
                 }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const bool has = j + u <= last;
-            const float wl = has ? __int_as_float(r[u].z) : 0.f;
-            const float wr = has ? __int_as_float(r[u].w) : 0.f;
+            const bool has = j + u < nrec;
+            const float wl = has ? rw[u].x : 0.f;
+            const float wr = has ? rw[u].y : 0.f;
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 fma_vec<BF16>(acc[v], t[u][0][v], make_float2(wl, wl));
@@ -191,25 +214,46 @@ __device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], cons
 // Backward of the gather: every record adds its two weighted taps of the cell's output gradient to the
 // feature gradient (the transpose of gather_list).  Vector reductions: texels are shared by cells.
 template <int V>
-__device__ __forceinline__ void scatter_list(const float4 (&go)[V], const bool (&on)[V], const int4 *list, int nrec,
-                                             float4 *const (&gfv)[V])
+__device__ __forceinline__ void scatter_list(const float4 (&go)[V], const bool (&on)[V], const int *loff, const float2 *lw, int nrec,
+                                             int rstep, float4 *const (&gfv)[V])
 {
     for (int j = 0; j < nrec; ++j) {
-        const int4 r = list[j];
-        const float wl = __int_as_float(r.z), wr = __int_as_float(r.w);
+        const int off = loff[j];
+        const float wl = lw[j].x, wr = lw[j].y;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             if (!on[v]) continue;  // ragged last channel block
-            if (wl != 0.f) atomicAdd(gfv[v] + r.x, make_float4(go[v].x * wl, go[v].y * wl, go[v].z * wl, go[v].w * wl));
-            if (wr != 0.f) atomicAdd(gfv[v] + r.y, make_float4(go[v].x * wr, go[v].y * wr, go[v].z * wr, go[v].w * wr));
+            if (wl != 0.f) atomicAdd(gfv[v] + off, make_float4(go[v].x * wl, go[v].y * wl, go[v].z * wl, go[v].w * wl));
+            if (wr != 0.f) atomicAdd(gfv[v] + off + rstep, make_float4(go[v].x * wr, go[v].y * wr, go[v].z * wr, go[v].w * wr));
         }
     }
 }
 
-// ---- step 1: one candidate column (cell c, camera n) -----------------------------------------------------
-// Returns false if no height bin of the column is valid; otherwise fills the descriptor (all but istart and the
-// first / last flags).
-__device__ __forceinline__ bool make_column(const KParams &p, const double *mats, const float *slope, const int *camfast,
+// ---- step 1a: can any height bin of candidate column (cell at xy, camera n) be valid? -------------------------
+// Every validity condition is a linear function of the height that must be positive (depth - 0.1; fx + 1/2 and
+// Wf - 1/2 - fx times the depth; likewise fy).  If one of them, relaxed by a texel, is negative at the first AND
+// the last bin centre it is negative in between: no bin of the column is valid.  NaN compares false: kept.
+__device__ __forceinline__ bool column_possible(const KParams &p, const double *m, double2 xy)
+{
+    const double zl = p.z_min + 0.5 * p.dz, zh = fma((double)(p.Z - 1), p.dz, zl);
+    const double a0 = fma(m[1], xy.y, fma(m[0], xy.x, m[3]));
+    const double a1 = fma(m[5], xy.y, fma(m[4], xy.x, m[7]));
+    const double a2 = fma(m[9], xy.y, fma(m[8], xy.x, m[11]));
+    const double dl = fma(m[10], zl, a2), dh = fma(m[10], zh, a2);
+    const double ul = fma(m[2], zl, a0), uh = fma(m[2], zh, a0);
+    const double vl = fma(m[6], zl, a1), vh = fma(m[6], zh, a1);
+    const double wf = (double)p.Wf + 0.5, hf = (double)p.Hf + 0.5;
+    bool out = (dl < 0.05) & (dh < 0.05);
+    out |= (fma(1.5, dl, ul) < 0.0) & (fma(1.5, dh, uh) < 0.0);   // fx < -3/2 wherever the depth is positive
+    out |= (fma(wf, dl, -ul) < 0.0) & (fma(wf, dh, -uh) < 0.0);   // fx > Wf + 1/2
+    out |= (fma(1.5, dl, vl) < 0.0) & (fma(1.5, dh, vh) < 0.0);
+    out |= (fma(hf, dl, -vl) < 0.0) & (fma(hf, dh, -vh) < 0.0);
+    return !out;
+}
+
+// ---- step 1b: the interval of valid bins of a column, exactly; affine form for height-independent cameras -----
+// Returns the number of valid bins (0: the column drops out) and fills D.
+__device__ __forceinline__ int column_build(const KParams &p, const double *mats, const float *slope, const int *camfast,
                                             double2 xy, int c, int n, ColDesc &D)
 {
     const double *m = mats + n * 12;
@@ -218,8 +262,9 @@ __device__ __forceinline__ bool make_column(const KParams &p, const double *mats
     const double a0 = fma(m[1], xy.y, fma(m[0], xy.x, m[3]));
     const double a1 = fma(m[5], xy.y, fma(m[4], xy.x, m[7]));
     const double a2 = fma(m[9], xy.y, fma(m[8], xy.x, m[11]));
-    const double wlim = (double)p.Wf - 0.5, hlim = (double)p.Hf - 0.5;
-
+    D.d0 = a0, D.d1 = a1, D.d2 = a2;
+    D.kk = 1;  // klo = 1 > khi = 0: no bins
+    D.meta = c | (n << 6);
     // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom -> conservative interval
     float lo = -1.f, hi = (float)p.Z;
     bool empty = false;
@@ -229,196 +274,391 @@ __device__ __forceinline__ bool make_column(const KParams &p, const double *mats
         else if (a <= 0.f) empty = true;  // independent of z (NaN: keep, tested exactly below)
     };
     const double d0 = fma(m[10], zc0, a2);
-    cond((float)(d0 - kDepthMin), sl[0]);
-    if (empty || !(lo < hi)) return false;
     const double p00 = fma(m[2], zc0, a0);
+    const double p10 = fma(m[6], zc0, a1);
+    cond((float)(d0 - kDepthMin), sl[0]);
     cond((float)p00, sl[1]);
     cond((float)fma((double)p.Wf, d0, -p00), sl[2]);
-    if (empty || !(lo < hi)) return false;
-    const double p10 = fma(m[6], zc0, a1);
     cond((float)p10, sl[3]);
     cond((float)fma((double)p.Hf, d0, -p10), sl[4]);
-    if (empty) return false;
+    if (empty || !(lo < hi)) return 0;
     // widen by a guard far above the float error, then confirm both ends exactly
     const float guard = 0.05f + 1e-5f * (float)p.Z;
     int klo = (int)floorf(fminf(fmaxf(lo - guard, -1.f), (float)p.Z)) + 1;
     int khi = (int)ceilf(fmaxf(fminf(hi + guard, (float)p.Z), -1.f)) - 1;
     klo = max(klo, 0);
     khi = min(khi, p.Z - 1);
+    const double wlim = (double)p.Wf - 0.5, hlim = (double)p.Hf - 0.5;
+    double fy_at = 0.0;  // fy of the bin tested last
     auto exact = [&](int k) {
         const double zw = fma((double)k, p.dz, zc0);
         const double d = fma(m[10], zw, a2);
         const double r = fast_rcp(d);  // d <= 0 or NaN gives inf / NaN: the tests below fail
         const double fx = fma(fma(m[2], zw, a0), r, -0.5);
         const double fy = fma(fma(m[6], zw, a1), r, -0.5);
+        fy_at = fy;
         return (d > kDepthMin) & (fx > -0.5) & (fx < wlim) & (fy > -0.5) & (fy < hlim);
     };
     while (klo <= khi && !exact(klo)) ++klo;
+    if (klo > khi) return 0;
+    const double fy_lo = fy_at;
     while (khi > klo && !exact(khi)) --khi;
-    if (klo > khi) return false;
-
-    const int nb = khi - klo + 1;
+    const bool rev = khi > klo && fy_at < fy_lo;  // rows ascend with the renumbered bins k' = khi - k
     D.kk = klo | (khi << 16);
-    D.pad0 = D.pad1 = 0;
-    D.istart = 0;
+    D.meta |= (rev ? 1 : 0) << 13;
     if (camfast[n]) {
         // depth and fx do not depend on the height: one texel column, fy affine in the bin index
         const double r = fast_rcp(a2);
         const double fx = fma(a0, r, -0.5);
         const double flx = floor(fx);
-        int xc;
-        fold_x((int)flx, (float)(fx - flx), p.Wf, xc, D.cl, D.cr);
-        const double ay = fma(p10, r, -0.5);   // fy of bin 0
-        const double sy = m[6] * p.dz * r;     // fy step per bin
-        const bool rev = sy < 0.0;
-        D.s = rev ? -sy : sy;
-        D.a = fma((double)(rev ? khi : klo), sy, ay);
-        const double fl0 = floor(D.a);
-        const double fln = floor(fma((double)(nb - 1), D.s, D.a));
-        const int nrows = (int)(fln - fl0) + 2;
-        const bool rows = p.reduce != FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM && nrows < nb && D.s >= 1e-9;
-        D.inv = rows ? (double)__frcp_rn((float)D.s) : 0.0;
-        D.offc = (n * p.Hf * p.Wf + xc) * p.vecs;
-        D.r0 = (int)fl0;
-        D.nitems = rows ? nrows : nb;
-        D.meta = c | (n << 8) | ((rows ? kKindRows : kKindBinsFast) << 16) | ((rev ? 1 : 0) << 18);
-    } else {
-        D.a = a0, D.s = a1, D.inv = a2;
-        D.offc = 0, D.r0 = 0, D.cl = D.cr = 0.f;
-        D.nitems = nb;
-        D.meta = c | (n << 8) | (kKindBinsGeneral << 16);
+        const int x0 = (int)flx;
+        const int edge = x0 < 0 ? 1 : (x0 >= p.Wf - 1 ? 2 : 0);
+        const int xc = edge == 1 ? 0 : (edge == 2 ? max(p.Wf - 2, 0) : x0);
+        const double sy = m[6] * p.dz * r;                 // fy step per bin
+        D.d0 = fma((double)(rev ? khi : klo), sy, fma(p10, r, -0.5));
+        D.d1 = rev ? -sy : sy;
+        D.f.offc = (n * p.Hf * p.Wf + xc) * p.vecs;
+        D.f.tx = (float)(fx - flx);
+        D.meta |= (1 << 12) | (edge << 14);
     }
-    return true;
+    return khi - klo + 1;
 }
 
-// ---- step 2: one item -> up to two row records -------------------------------------------------------------
-struct ItemOut {
-    bool va, vb;
-    int4 ra, rb;
-};
+// An affine column with a step of at most two rows per bin touches every texel row from its first bin's row to the
+// row below its last bin's row: its records are those rows (inside the map), one each, and a run is a range of
+// ROWS.  With larger steps the rows of successive bins never coincide: two records per bin, and a run is a range
+// of BINS.  Either way the number of records of a run is known without walking it.
+__device__ __forceinline__ bool affine_by_rows(const ColDesc &D) { return D.d1 <= 1.999; }
 
-__device__ __forceinline__ void make_item(const KParams &p, const WarpSmem &sm, const double *mats, const ColDesc &D, int li,
-                                          ItemOut &o)
+// Units (rows or bins) of an affine column that its runs are cut from, and the first row it writes.
+__device__ __forceinline__ int affine_units(const KParams &p, const ColDesc &D, int nb, int &row_first)
 {
-    o.va = o.vb = false;
-    const int kind = (D.meta >> 16) & 3;
-    const int klo = D.kk & 0xffff, khi = D.kk >> 16, nb = khi - klo + 1;
-    const int rowv = p.Wf * p.vecs;
-    if (kind == kKindRows) {
-        // texel row r of a height-independent column: the bins k' with floor(a + k' s) == r are k' in [k1, k2),
-        // those of the row above [k0, k1); their (1 - ty) and ty sums are arithmetic series
-        const int r = D.r0 + li;
-        const double ay = D.a, sy = D.s, inv = D.inv;
-        auto first_bin_at = [&](double rr) {  // smallest k' in [0, nb] with a + k' s >= rr
-            double e = ceil((rr - ay) * inv);
+    const int r_first = (int)floor(D.d0), r_last = (int)floor(fma((double)(nb - 1), D.d1, D.d0));
+    row_first = max(r_first, 0);
+    return affine_by_rows(D) ? max(0, min(r_last + 1, p.Hf - 1) - row_first + 1) : nb;
+}
+
+// Records of a run of an affine column: [u0, u0 + len) are rows counted from the column's first written row, or bins.
+__device__ __forceinline__ int affine_run_records(const KParams &p, const ColDesc &D, int u0, int len)
+{
+    if (affine_by_rows(D)) return len;
+    const int r_first = (int)floor(fma((double)u0, D.d1, D.d0)), r_last = (int)floor(fma((double)(u0 + len - 1), D.d1, D.d0));
+    return 2 * len - (r_first < 0 ? 1 : 0) - (r_last + 1 > p.Hf - 1 ? 1 : 0);
+}
+
+// ---- step 2: walker of an affine column.  Writes exactly affine_run_records() records. -------------------------
+// A run of rows [ra, rb) takes the bins whose upper tap lies in rows ra - 1 .. rb - 1: a row's weight is the (1 - ty)
+// of the bins in it plus the ty of the bins in the row above, so every run is complete by itself and neighbouring
+// runs share no record.
+__device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm, const ColDesc &D, int u0, int len,
+                                            int *out_off, float2 *out_w, int cap)
+{
+    const int meta = D.meta;
+    const bool rev = (meta >> 13) & 1;
+    const int edge = (meta >> 14) & 3;
+    const float tx = D.f.tx;
+    float cl = 0.f, cr = 0.f;  // horizontal weights of the two loaded texels (an out-of-map tap weighs 0)
+    if (edge == 0) cl = 1.f - tx, cr = tx;
+    else if (edge == 1) cl = tx;
+    else if (p.Wf > 1) cr = 1.f - tx;
+    else cl = 1.f - tx;
+    const bool eq1 = p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM;
+    const int klo = D.kk & 0xffff, khi = (D.kk >> 16) & 0xffff, nb = khi - klo + 1;
+    const unsigned char *den = sm.den + (meta & 63) * p.Z + (rev ? khi : klo);  // den[cell][bin of k' = 0]
+    const int dstep = rev ? -1 : 1;
+    const int rowv = p.Wf * p.vecs, offc = D.f.offc;
+    const double S = D.d1, A = D.d0;
+    const bool by_rows = affine_by_rows(D);
+
+    int kb = u0, ke = u0 + len;  // bins [kb, ke)
+    int ra = 0, rb = p.Hf;       // rows written: [ra, rb)
+    if (by_rows) {
+        ra = max((int)floor(A), 0) + u0, rb = ra + len;
+        const double inv = (double)__frcp_rn((float)S);
+        auto first_bin_at = [&](double rr) {  // smallest k' in [0, nb] with A + k' S >= rr
+            double e = ceil((rr - A) * inv);
             e = fmin(fmax(e, 0.0), (double)nb);  // NaN -> 0
             int k = (int)e;
-            if (k > 0 && fma((double)(k - 1), sy, ay) >= rr) --k;
-            else if (k < nb && fma((double)k, sy, ay) < rr) ++k;
+            if (k > 0 && fma((double)(k - 1), S, A) >= rr) --k;
+            else if (k < nb && fma((double)k, S, A) < rr) ++k;
             return k;
         };
-        const double rr = (double)r;
-        const int k0 = first_bin_at(rr - 1.0), k1 = first_bin_at(rr), k2 = first_bin_at(rr + 1.0);
-        const double dm = (double)(k1 - k0), dn = (double)(k2 - k1);
-        const double sum_ty_row = fma(dn, ay - rr, sy * (0.5 * dn * (double)(k1 + k2 - 1)));          // over [k1, k2)
-        const double sum_ty_above = fma(dm, ay - (rr - 1.0), sy * (0.5 * dm * (double)(k0 + k1 - 1)));  // over [k0, k1)
-        const float w = (float)((dn - sum_ty_row) + sum_ty_above);
-        if (r >= 0 && r <= p.Hf - 1 && w != 0.f) {
-            const int off = FB_IDX(D.offc + r * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
-            o.va = true;
-            o.ra = make_int4(off, off + p.rstep, __float_as_int(D.cl * w), __float_as_int(D.cr * w));
+        kb = first_bin_at((double)(ra - 1)), ke = first_bin_at((double)rb);
+    }
+    int n = 0;
+    auto emit = [&](int row, float w) {
+        if (row >= ra && row < rb) {
+            const int at = by_rows ? row - ra : n;
+            if (at < cap) {
+                out_off[at] = FB_IDX(offc + row * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
+                out_w[at] = make_float2(cl * w, cr * w);
+            }
+            ++n;
         }
+    };
+    if (kb >= ke) {  // (cannot happen: a run of rows always has bins, a run of bins has len >= 1; leave no stale weights)
+        for (int i = 0; i < min(len, cap); ++i) out_off[i] = offc, out_w[i] = make_float2(0.f, 0.f);
         return;
     }
+    double kd = (double)kb;
+    int ro;
+    float wu, wl;
+    {
+        const double fy = fma(kd, S, A), fl = floor(fy);
+        const float ty = (float)(fy - fl);
+        const float s = eq1 ? 1.f / (float)max(1, (int)den[kb * dstep]) : 1.f;
+        ro = (int)fl;
+        wu = (1.f - ty) * s, wl = ty * s;
+    }
+    for (int k = kb + 1; k < ke; ++k) {
+        kd += 1.0;
+        const double fy = fma(kd, S, A), fl = floor(fy);
+        const int r = (int)fl;
+        const float ty = (float)(fy - fl);
+        const float s = eq1 ? 1.f / (float)max(1, (int)den[k * dstep]) : 1.f;
+        if (r != ro) {
+            emit(ro, wu);
+            if (!by_rows || r != ro + 1) {
+                emit(ro + 1, wl);
+                wl = 0.f;
+            }
+            wu = wl, wl = 0.f, ro = r;
+        }
+        wu = fmaf(1.f - ty, s, wu);
+        wl = fmaf(ty, s, wl);
+    }
+    emit(ro, wu);
+    emit(ro + 1, wl);
+}
 
-    const bool general = kind == kKindBinsGeneral;
-    const bool rev = (D.meta >> 18) & 1;
-    const int cell = D.meta & 0xff, cam = (D.meta >> 8) & 0xff;
+// ---- step 2: walker of a general column (every bin projected in fp64).  COUNT-only or EMIT. ------------------------
+template <bool EMIT>
+__device__ __forceinline__ int walk_general(const KParams &p, const WarpSmem &sm, const double *mats, const ColDesc &D, int k0,
+                                            int len, int *out_off, float2 *out_w, int cap)
+{
+    const int meta = D.meta;
+    const bool rev = (meta >> 13) & 1;
+    const int cell = meta & 63, cam = (meta >> 6) & 63;
+    const int klo = D.kk & 0xffff, khi = (D.kk >> 16) & 0xffff;
+    const int rowv = p.Wf * p.vecs;
     const double *m = mats + cam * 12;
     const double zc0 = p.z_min + 0.5 * p.dz;
-    auto eval = [&](int kp, Tap &t) {
-        if (general) {
-            const double zw = fma((double)(klo + kp), p.dz, zc0);
-            const double d = fma(m[10], zw, D.inv);
-            const double r = fast_rcp(d);
-            const double fx = fma(fma(m[2], zw, D.a), r, -0.5);
-            const double fy = fma(fma(m[6], zw, D.s), r, -0.5);
-            const double flx = floor(fx), fly = floor(fy);
-            t.x0 = (int)flx;
-            t.y0 = (int)fly;
-            t.ty = (float)(fy - fly);
-            fold_x(t.x0, (float)(fx - flx), p.Wf, t.xc, t.cl, t.cr);
-        } else {
-            const double fy = fma((double)kp, D.s, D.a);
-            const double fly = floor(fy);
-            t.x0 = 0, t.xc = 0;
-            t.y0 = (int)fly;
-            t.ty = (float)(fy - fly);
-            t.cl = D.cl, t.cr = D.cr;
+    int n = 0;
+    bool open = false;
+    int ro = 0, xo = 0, xco = 0;  // open rows (ro, ro + 1) at bilinear corner column xo, first loaded texel xco
+    float uL = 0.f, uR = 0.f, lL = 0.f, lR = 0.f;
+    auto put = [&](int row, float wl, float wr) {
+        if (row >= 0 && row <= p.Hf - 1) {
+            if (EMIT && n < cap) {
+                const int off = FB_IDX((cam * p.Hf * p.Wf + xco) * p.vecs + row * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
+                out_off[n] = off, out_w[n] = make_float2(wl, wr);
+            }
+            ++n;
         }
     };
-    auto scale = [&](int kp) {  // Eq. 1: 1 / max(1, cameras that see this cell at this height)
-        if (p.reduce != FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) return 1.f;
-        const int k = rev ? khi - kp : klo + kp;
-        const unsigned dn = sm.den[FB_IDX(cell * p.Z + k, p.den_bytes, p.err)];
-        return 1.f / (float)(dn > 1u ? dn : 1u);
-    };
-
-    Tap cur, pv;
-    eval(li, cur);
-    bool head = true;
-    if (li > 0) {
-        eval(li - 1, pv);
-        head = !(pv.x0 == cur.x0 && pv.y0 == cur.y0);
-    }
-    if (!head) return;  // the lane that starts this run of bins covers it
-    float uL = 0.f, uR = 0.f, lL = 0.f, lR = 0.f;
-    bool next_continues = false;  // the next run starts on this run's lower row: its record takes our lower weights
-    {
-        int e = li;
-        Tap t = cur;
-        while (true) {
-            const float s = scale(e);
-            const float wy1 = t.ty * s, wy0 = (1.f - t.ty) * s;
-            uL = fmaf(t.cl, wy0, uL), uR = fmaf(t.cr, wy0, uR);
-            lL = fmaf(t.cl, wy1, lL), lR = fmaf(t.cr, wy1, lR);
-            if (++e >= nb) break;
-            eval(e, t);
-            if (!(t.x0 == cur.x0 && t.y0 == cur.y0)) {
-                next_continues = t.x0 == cur.x0 && t.y0 == cur.y0 + 1;
-                break;
+    for (int i0 = 0; i0 < len; i0 += kWalkIlp) {
+        int r[kWalkIlp], x0[kWalkIlp], xc[kWalkIlp];
+        float cl[kWalkIlp], cr[kWalkIlp], ty[kWalkIlp];
+#pragma unroll
+        for (int i = 0; i < kWalkIlp; ++i) {
+            const int kp = k0 + min(i0 + i, len - 1);  // past the end: the last bin again (ignored below)
+            const double zw = fma((double)(rev ? khi - kp : klo + kp), p.dz, zc0);
+            const double d = fma(m[10], zw, D.d2);
+            const double rd = fast_rcp(d);
+            const double fx = fma(fma(m[2], zw, D.d0), rd, -0.5);
+            const double fy = fma(fma(m[6], zw, D.d1), rd, -0.5);
+            const double flx = floor(fx), fly = floor(fy);
+            r[i] = (int)fly, x0[i] = (int)flx;
+            ty[i] = (float)(fy - fly);
+            fold_x(x0[i], (float)(fx - flx), p.Wf, xc[i], cl[i], cr[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < kWalkIlp; ++i) {
+            if (i0 + i < len) {
+                const bool col_same = open & (x0[i] == xo);
+                const bool same = col_same & (r[i] == ro), next = col_same & (r[i] == ro + 1);
+                if (!same) {
+                    if (open) {
+                        put(ro, uL, uR);
+                        if (!next) put(ro + 1, lL, lR);
+                    }
+                    uL = next ? lL : 0.f, uR = next ? lR : 0.f, lL = 0.f, lR = 0.f;
+                    ro = r[i], xo = x0[i], xco = xc[i], open = true;
+                }
+                if (EMIT) {
+                    float s = 1.f;
+                    if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {  // Eq. 1: 1 / max(1, cameras that see this height)
+                        const int kp = k0 + i0 + i;
+                        const unsigned dn = sm.den[FB_IDX(cell * p.Z + (rev ? khi - kp : klo + kp), p.den_bytes, p.err)];
+                        s = 1.f / (float)(dn > 1u ? dn : 1u);
+                    }
+                    const float wy1 = ty[i] * s, wy0 = (1.f - ty[i]) * s;
+                    uL = fmaf(cl[i], wy0, uL), uR = fmaf(cr[i], wy0, uR);
+                    lL = fmaf(cl[i], wy1, lL), lR = fmaf(cr[i], wy1, lR);
+                }
             }
         }
     }
-    if (li > 0 && pv.x0 == cur.x0 && pv.y0 + 1 == cur.y0) {
-        // the run before ended one row above: its lower-row weights belong to our upper row
-        int b = li - 1;
-        Tap t = pv;
-        while (true) {
-            const float wy1 = t.ty * scale(b);
-            uL = fmaf(t.cl, wy1, uL), uR = fmaf(t.cr, wy1, uR);
-            if (--b < 0) break;
-            eval(b, t);
-            if (!(t.x0 == pv.x0 && t.y0 == pv.y0)) break;
+    if (open) {
+        put(ro, uL, uR);
+        put(ro + 1, lL, lR);
+    }
+    return n;
+}
+
+// The three geometry steps are separate functions (not inlined) so that their fp64-heavy register needs stay out of
+// the gather loop's allocation; everything they exchange lives in the warp's shared memory.
+struct WarpCtx {
+    const double *mats;
+    const float *slope;
+    const int *camfast;
+    unsigned char *warp_base;  // this warp's shared memory
+};
+
+__device__ __forceinline__ WarpSmem warp_smem(const KParams &p, unsigned char *warp_base)
+{
+    WarpSmem sm;
+    warp_smem_layout(warp_base, &sm, p.slots, p.colcap, p.wcap, p.ct, p.ct * p.N, p.den_bytes);
+    return sm;
+}
+
+// ---- step 1a over a super-block: candidates -> survivors, compacted in (cell, camera) order.  Returns their number.
+__device__ __forceinline__ int survey_candidates(const KParams &p, WarpCtx cx, unsigned in_mask)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const WarpSmem sm = warp_smem(p, cx.warp_base);
+    const int lane = threadIdx.x & 31;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const int ncand = p.ct * p.N;
+    int nsurv = 0;
+    for (int p0 = 0; p0 < ncand; p0 += 32) {
+        const int pr = p0 + lane;
+        const int c = (int)(((float)pr + 0.5f) * p.inv_n), n = pr - c * p.N;
+        bool keep = false;
+        if (pr < ncand && ((in_mask >> c) & 1u)) keep = column_possible(p, cx.mats + n * 12, sm.cellxy[c]);
+        const unsigned bal = __ballot_sync(FULL, keep);
+        const int idx = nsurv + __popc(bal & lt_mask);
+        if (pr < ncand && n == 0) sm.cfirst[FB_IDX(c, kMaxCt + 1, p.err)] = idx;  // where the cell's columns start
+        if (keep) sm.cand[FB_IDX(idx, ncand, p.err)] = (uint16_t)(c | (n << 8));
+        nsurv += __popc(bal);
+    }
+    if (lane == 0) sm.cfirst[p.ct] = nsurv;
+    __syncwarp();
+    return nsurv;
+}
+
+// ---- step 1b over a segment (survivors [jb, jb + ncols), cells [c_lo, c_hi)): exact intervals, runs and their record
+// counts (two exclusive scans over the columns), valid samples per cell, Eq. 1 camera counts.  Returns the number of runs.
+__device__ __forceinline__ int build_columns(const KParams &p, WarpCtx cx, int jb, int ncols, int c_lo, int c_hi)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const WarpSmem sm = warp_smem(p, cx.warp_base);
+    const int lane = threadIdx.x & 31;
+    int nw = 0, nrec_seg = 0;
+    for (int j0 = 0; j0 < ncols; j0 += 32) {
+        const int j = j0 + lane;
+        ColDesc D;
+        int nb = 0;
+        if (j < ncols) {
+            const int cn = sm.cand[jb + j];
+            nb = column_build(p, cx.mats, cx.slope, cx.camfast, sm.cellxy[cn & 0xff], cn & 0xff, cn >> 8, D);
+            sm.col[FB_IDX(j, p.colcap, p.err)] = D;
+        }
+        bool affine = false;
+        int units = nb, row_first = 0;  // what the column's runs are cut from: bins, or rows of an affine column
+        if (nb > 0) {
+            affine = (D.meta >> 12) & 1;
+            if (affine) units = affine_units(p, D, nb, row_first);
+        }
+        const int runs = (units + p.walk - 1) / p.walk;
+        int x = runs;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int y = __shfl_up_sync(FULL, x, off);
+            if (lane >= off) x += y;
+        }
+        const int wbase = nw + x - runs;
+        nw += __shfl_sync(FULL, x, 31);
+        int mine = 0;  // records of this lane's column
+        if (j < ncols) {
+            sm.colw[j] = wbase;
+            for (int i = 0; i < runs; ++i) {
+                const int u0 = i * p.walk, len = min(p.walk, units - u0);
+                sm.wk[FB_IDX(wbase + i, p.wcap, p.err)] = (uint32_t)j | ((uint32_t)u0 << 8) | ((uint32_t)(len - 1) << 24);
+                sm.woff[FB_IDX(wbase + i, p.wcap + 1, p.err)] = mine;
+                mine += affine ? affine_run_records(p, D, u0, len) : walk_general<false>(p, sm, cx.mats, D, u0, len, nullptr, nullptr, 0);
+            }
+        }
+        int y = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int z = __shfl_up_sync(FULL, y, off);
+            if (lane >= off) y += z;
+        }
+        const int rbase = nrec_seg + y - mine;
+        nrec_seg += __shfl_sync(FULL, y, 31);
+        if (j < ncols)
+            for (int i = 0; i < runs; ++i) sm.woff[wbase + i] += rbase;
+    }
+    if (lane == 0) sm.colw[ncols] = nw, sm.woff[nw] = nrec_seg;
+    __syncwarp();
+
+    // valid samples per cell; Eq. 1: cameras per (cell, height bin) -- the intervals say it all
+    if (lane >= c_lo && lane < c_hi) {
+        int n = 0;
+        for (int j = sm.cfirst[lane] - jb; j < sm.cfirst[lane + 1] - jb; ++j) {
+            const int kk = sm.col[j].kk;
+            n += max(0, ((kk >> 16) & 0xffff) - (kk & 0xffff) + 1);
+        }
+        sm.cnt[lane] = n;
+    }
+    if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
+        for (int i = c_lo * p.Z + lane; i < c_hi * p.Z; i += 32) {
+            const int c = i / p.Z, k = i - c * p.Z;
+            int dn = 0;
+            for (int j = sm.cfirst[c] - jb; j < sm.cfirst[c + 1] - jb; ++j) {
+                const int kk = sm.col[j].kk;
+                dn += (k >= (kk & 0xffff) && k <= ((kk >> 16) & 0xffff)) ? 1 : 0;
+            }
+            sm.den[FB_IDX(i, p.den_bytes, p.err)] = (unsigned char)dn;
         }
     }
-    const int offc = general ? (cam * p.Hf * p.Wf + cur.xc) * p.vecs : D.offc;
-    const int r = cur.y0;
-    if (r >= 0 && r <= p.Hf - 1 && (uL != 0.f || uR != 0.f)) {
-        const int off = FB_IDX(offc + r * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
-        o.va = true;
-        o.ra = make_int4(off, off + p.rstep, __float_as_int(uL), __float_as_int(uR));
+    __syncwarp();
+    return nw;
+}
+
+// ---- step 2: a round.  As many runs from `wa` on as fit the record slots are walked, one lane each; returns the
+// first run not taken.
+__device__ FB_EMIT_INLINE int emit_round(const KParams &p, WarpCtx cx, int wa, int nw)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const WarpSmem sm = warp_smem(p, cx.warp_base);
+    const int lane = threadIdx.x & 31;
+    __syncwarp();
+    const int base = sm.woff[wa];
+    int wb = wa;
+    for (int w0 = wa + 1; w0 <= nw; w0 += 32) {
+        const int w = w0 + lane;
+        const bool fits = w <= nw && sm.woff[w] - base <= p.slots;
+        const unsigned bal = __ballot_sync(FULL, fits);
+        wb = w0 - 1 + __popc(bal);
+        if (bal != FULL) break;
     }
-    if (!next_continues && r + 1 >= 0 && r + 1 <= p.Hf - 1 && (lL != 0.f || lR != 0.f)) {
-        const int off = FB_IDX(offc + (r + 1) * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
-        o.vb = true;
-        o.rb = make_int4(off, off + p.rstep, __float_as_int(lL), __float_as_int(lR));
+    if (wb <= wa) wb = wa + 1;  // (cannot happen: one run always fits; never loop without progress)
+    for (int w = wa + lane; w < wb && !(p.dbg & 2); w += 32) {
+        const uint32_t wd = sm.wk[w];
+        const ColDesc D = sm.col[FB_IDX(wd & 0xff, p.colcap, p.err)];
+        const int at = FB_IDX(sm.woff[w] - base, p.slots, p.err);
+        if ((D.meta >> 12) & 1) walk_affine(p, sm, D, (wd >> 8) & 0xffff, (wd >> 24) + 1, sm.roff + at, sm.rw + at, p.slots - at);
+        else walk_general<true>(p, sm, cx.mats, D, (wd >> 8) & 0xffff, (wd >> 24) + 1, sm.roff + at, sm.rw + at, p.slots - at);
     }
+    __syncwarp();
+    return wb;
 }
 
 // WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
 template <int V, bool BF16, int WARPS, bool BWD, bool WIDE>
-__global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : 20) / WARPS)
+__global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / WARPS)
     vt_tiled_kernel(const KParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -426,20 +666,19 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : 20) / WARPS)
     constexpr int THREADS = WARPS * 32;
     constexpr unsigned FULL = 0xffffffffu;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const unsigned lt_mask = (1u << lane) - 1u;
     const int b = blockIdx.z;
 
     double *mats = reinterpret_cast<double *>(smem_raw);
     float *slope = reinterpret_cast<float *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)));
-    int *camfast = reinterpret_cast<int *>(smem_raw + align16((size_t)p.N * 12 * sizeof(double)) +
-                                           align16((size_t)p.N * 5 * sizeof(float)));
-    WarpSmem sm;
-    {
-        const size_t per_warp = warp_smem_layout(nullptr, nullptr, p.slots, p.ncap, p.den_bytes);
-        warp_smem_layout(smem_raw + cta_table_bytes(p.N) + warp * per_warp, &sm, p.slots, p.ncap, p.den_bytes);
-    }
+    int *camfast = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(slope) + align16((size_t)p.N * 5 * sizeof(float)));
+    int *celltab = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(camfast) + align16((size_t)p.N * sizeof(int)));
+    WarpCtx cx;
+    cx.mats = mats, cx.slope = slope, cx.camfast = camfast;
+    cx.warp_base = smem_raw + align16(cta_table_bytes(p.N)) +
+                   warp * warp_smem_layout(nullptr, nullptr, p.slots, p.colcap, p.wcap, p.ct, p.ct * p.N, p.den_bytes);
+    const WarpSmem sm = warp_smem(p, cx.warp_base);
 
-    // ---- per-CTA tables: camera matrices (scaled to feature texels), condition slopes, camera class
+    // ---- per-CTA tables: camera matrices (scaled to feature texels), condition slopes, camera class, cell positions
     for (int i = tid; i < p.N * 12; i += THREADS) {
         const int n = i / 12, e = i - n * 12;
         double v = (double)__ldg(p.l2i + ((size_t)b * p.N + n) * 16 + e);
@@ -458,8 +697,18 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : 20) / WARPS)
         slope[n * 5 + 4] = (float)(((double)p.Hf * m10 - m6) * p.dz);
         camfast[n] = (m10 == 0.0 && m2 == 0.0) ? 1 : 0;
     }
-    // every record slot always holds loadable offsets: lanes may read (not use) slots past their list
-    for (int i = lane; i < p.slots; i += 32) sm.rec[i] = make_int4(0, 0, 0, 0);
+    for (int c = tid; c < kMaxCt; c += THREADS) {
+        int v = 0;
+        if (c < p.ct) {
+            const int s = c / p.cpw, j = c - s * p.cpw;  // sub-block, cell inside it
+            const int si = s / p.sby, sj = s - si * p.sby;
+            const int jx = j / p.wy, jy = j - jx * p.wy;
+            v = (si * p.wx + jx) | ((sj * p.wy + jy) << 8);
+        }
+        celltab[c] = v;
+    }
+    // every record slot always holds loadable offsets: the gather may read (not use) slots past a list
+    for (int i = lane; i < p.slots + 4; i += 32) sm.roff[i] = 0, sm.rw[i] = make_float2(0.f, 0.f);
     __syncthreads();  // the only CTA-wide barrier
 
     // ---- gather role of this lane inside a sub-block
@@ -480,199 +729,123 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : 20) / WARPS)
             gfv[v] = BWD ? reinterpret_cast<float4 *>(p.gfeat) + cam0 + vi : nullptr;
         }
     }
-    const int ncand = p.cpw * p.N;
+    const int my_tab = celltab[lane];
 
     for (int rep = 0; rep < p.reps; ++rep) {
-        // ---- which sub-block: ids run along y inside bands of `band` rows of sub-blocks
+        // ---- which super-block: ids run along y inside bands of `band` rows of super-blocks
         const int id = (blockIdx.x * WARPS + warp) * p.reps + rep;
         const int per_band = p.band * p.blocks_y;
         const int bandi = id / per_band, rem = id - bandi * per_band;
         const int by = rem / p.band, bx = bandi * p.band + (rem - by * p.band);
         if (bx >= p.blocks_x) continue;  // warp-uniform
-        const int ix0 = bx * p.wx, iy0 = by * p.wy;
+        const int ix0 = bx * (p.sbx * p.wx), iy0 = by * (p.sby * p.wy);
 
-        unsigned in_mask;  // bit c: cell c of the sub-block is inside the grid
+        unsigned in_mask;  // bit c: cell c of the super-block is inside the grid
         {
-            const int lx = lane / p.wy, ly = lane - lx * p.wy;
-            const bool in = (lane < p.cpw) && (ix0 + lx < p.X) && (iy0 + ly < p.Y);
-            if (lane < kMaxCells) {
-                const double nan = __longlong_as_double(0x7ff8000000000000LL);
+            const int lx = my_tab & 0xff, ly = my_tab >> 8;
+            const bool in = (lane < p.ct) && (ix0 + lx < p.X) && (iy0 + ly < p.Y);
+            const double nan = __longlong_as_double(0x7ff8000000000000LL);
+            if (lane < p.ct)
                 sm.cellxy[lane] = make_double2(in ? p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx : nan,
                                                in ? p.y_min + ((double)(iy0 + ly) + 0.5) * p.dy : nan);
-            }
             in_mask = __ballot_sync(FULL, in);
         }
         __syncwarp();
+        survey_candidates(p, cx, in_mask);
 
-        // ---- step 1: columns, compacted in (cell, camera) order
-        int ncols = 0;
-        for (int p0 = 0; p0 < ncand; p0 += 32) {
-            const int pr = p0 + lane;
-            const int c = pr / p.N, n = pr - c * p.N;
-            ColDesc D;
-            bool valid = false;
-            if (pr < ncand && ((in_mask >> c) & 1u)) valid = make_column(p, mats, slope, camfast, sm.cellxy[c], c, n, D);
-            const unsigned bal = __ballot_sync(FULL, valid);
-            const int idx = ncols + __popc(bal & lt_mask);
-            if (pr < ncand && n == 0) sm.cfirst[FB_IDX(c, kMaxCells + 1, p.err)] = idx;  // where the cell's columns start
-            if (valid) sm.col[FB_IDX(idx, p.ncap, p.err)] = D;
-            ncols += __popc(bal);
-        }
-        if (lane == 0) sm.cfirst[p.cpw] = ncols;
-        __syncwarp();
+        // ---- segments: as many sub-blocks as have at most `colcap` surviving columns together (normally all of them)
+        for (int s0 = 0; s0 < p.sbn;) {
+            const int jb = sm.cfirst[s0 * p.cpw];
+            int s1 = s0 + 1;
+            while (s1 < p.sbn && sm.cfirst[min((s1 + 1) * p.cpw, p.ct)] - jb <= p.colcap) ++s1;
+            const int ncols = sm.cfirst[min(s1 * p.cpw, p.ct)] - jb;  // <= colcap: a sub-block has at most cpw * N candidates
+            const int nw = (p.dbg & 4) ? 0 : build_columns(p, cx, jb, ncols, s0 * p.cpw, min(s1 * p.cpw, p.ct));
 
-        // ---- item offsets of the columns (exclusive scan), first / last column of a cell, valid samples per cell
-        int T = 0;
-        for (int j0 = 0; j0 < ncols; j0 += 32) {
-            const int j = j0 + lane;
-            const int ni = j < ncols ? sm.col[j].nitems : 0;
-            int x = ni;
+            // ---- rounds of runs [wa, wb) that fit the record slots; gather sub-block by sub-block
+            int wa = 0, wb = 0;
+            for (int s = s0; s < s1; ++s) {
+                const int cell = s * p.cpw + (role ? cg : 0);
+                const bool lane_on = role && ((in_mask >> cell) & 1u);
+                const int tab = celltab[cell];
+                // (lanes without a cell inside the grid never use it)
+                const size_t ocell = lane_on ? (size_t)FB_IDX(((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8)),
+                                                              (size_t)p.B * p.X * p.Y, p.err) : 0;
+                int sw_lo = sm.colw[sm.cfirst[s * p.cpw] - jb], sw_hi = sm.colw[sm.cfirst[min((s + 1) * p.cpw, p.ct)] - jb];
+                int cw_lo = sm.colw[sm.cfirst[cell] - jb], cw_hi = sm.colw[sm.cfirst[cell + 1] - jb];  // this lane's cell
+                if (p.dbg & 4) sw_lo = sw_hi = cw_lo = cw_hi = 0;
+                int pos = sw_lo;  // runs of this sub-block before `pos` are done
+                if (pos < sw_hi && pos >= wb) wa = pos, wb = emit_round(p, cx, wa, nw);  // (no accumulator is live here)
+
+                float2 acc[V][PV];
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int y = __shfl_up_sync(FULL, x, off);
-                if (lane >= off) x += y;
-            }
-            if (j < ncols) {
-                const int meta = sm.col[j].meta, c = meta & 0xff;
-                sm.col[j].istart = T + x - ni;
-                sm.col[j].meta = meta | ((j == sm.cfirst[c]) ? (1 << 19) : 0) | ((j + 1 == sm.cfirst[c + 1]) ? (1 << 20) : 0);
-            }
-            T += __shfl_sync(FULL, x, 31);
-        }
-        if (lane < p.cpw) {
-            int n = 0;
-            for (int j = sm.cfirst[lane]; j < sm.cfirst[lane + 1]; ++j) {
-                const int kk = sm.col[j].kk;
-                n += (kk >> 16) - (kk & 0xffff) + 1;
-            }
-            sm.cnt[lane] = n;
-        }
-        if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
-            // cameras per (cell, height bin): the columns' intervals say it all
-            for (int i = lane; i < p.cpw * p.Z; i += 32) {
-                const int c = i / p.Z, k = i - c * p.Z;
-                int dn = 0;
-                for (int j = sm.cfirst[c]; j < sm.cfirst[c + 1]; ++j) {
-                    const int kk = sm.col[j].kk;
-                    dn += (k >= (kk & 0xffff) && k <= (kk >> 16)) ? 1 : 0;
-                }
-                sm.den[FB_IDX(i, p.den_bytes, p.err)] = (unsigned char)dn;
-            }
-        }
-        __syncwarp();
-
-        float2 acc[V][PV];
+                for (int v = 0; v < V; ++v)
 #pragma unroll
-        for (int v = 0; v < V; ++v)
+                    for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
+                float4 go[V];  // backward: this lane's channel vectors of the cell's output gradient
+                bool on[V];
+                if (BWD) {
+                    const int count = sm.cnt[cell];
+                    const float gscale = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
 #pragma unroll
-            for (int e = 0; e < PV; ++e) acc[v][e] = make_float2(0.f, 0.f);
-
-        const int cell = role ? cg : 0;
-        const bool lane_on = role && ((in_mask >> cell) & 1u);
-        const int my_lx = cell / p.wy, my_ly = cell - my_lx * p.wy;
-        // (lanes without a cell inside the grid never use it)
-        const size_t ocell = lane_on ? (size_t)FB_IDX(((size_t)b * p.X + (ix0 + my_lx)) * p.Y + (iy0 + my_ly),
-                                                      (size_t)p.B * p.X * p.Y, p.err) : 0;
-
-        float4 go[V];  // backward: this lane's channel vectors of the cell's output gradient
-        bool on[V];
-        if (BWD) {
-            const int count = sm.cnt[cell];
-            const float gscale = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int vi = vec0 + v * vstep;
-                go[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                on[v] = lane_on && vi < p.vecs;
-                if (on[v] && T > 0) {
-                    go[v] = __ldg(reinterpret_cast<const float4 *>(p.gout + ocell * p.C) + vi);
-                    go[v].x *= gscale, go[v].y *= gscale, go[v].z *= gscale, go[v].w *= gscale;
-                }
-            }
-        }
-
-        // ---- rounds: fill the record list from the items in order, then gather it
-        int t0 = 0;
-        while (t0 < T) {
-            if (lane < kMaxCells) sm.cstart[lane] = 0, sm.cend[lane] = 0;
-            __syncwarp();
-            const int round_first = t0;
-            int fill = 0;
-            while (t0 < T && fill + 64 <= p.slots) {
-                const int t = t0 + lane;
-                const int pass_last = min(T, t0 + 32) - 1;
-                ItemOut o;
-                o.va = o.vb = false;
-                int q = 0, li = 0, meta = 0, nitems = 0;
-                if (t < T) {
-                    int lo = 0, hi = ncols;  // istart[lo] <= t < istart[hi]
-                    while (hi - lo > 1) {
-                        const int mid = (lo + hi) >> 1;
-                        if (sm.col[mid].istart <= t) lo = mid;
-                        else hi = mid;
-                    }
-                    const ColDesc D = sm.col[FB_IDX(lo, p.ncap, p.err)];
-                    li = t - D.istart;
-                    meta = D.meta, nitems = D.nitems;
-                    q = meta & 0xff;
-                    make_item(p, sm, mats, D, li, o);
-                }
-                const unsigned ba = __ballot_sync(FULL, o.va), bb = __ballot_sync(FULL, o.vb);
-                const int pos_a = fill + __popc(ba & lt_mask) + __popc(bb & lt_mask);
-                const int pos_b = pos_a + (o.va ? 1 : 0);
-                if (o.va) sm.rec[FB_IDX(pos_a, p.slots, p.err)] = o.ra;
-                if (o.vb) sm.rec[FB_IDX(pos_b, p.slots, p.err)] = o.rb;
-                if (t < T) {
-                    if ((li == 0 && (meta & (1 << 19))) || t == round_first) sm.cstart[FB_IDX(q, kMaxCells, p.err)] = pos_a;
-                    if ((li == nitems - 1 && (meta & (1 << 20))) || t == pass_last)
-                        sm.cend[FB_IDX(q, kMaxCells, p.err)] = pos_b + (o.vb ? 1 : 0);
-                }
-                fill += __popc(ba) + __popc(bb);
-                t0 += 32;
-                __syncwarp();
-            }
-            if (t0 > T) t0 = T;
-
-            const int c0 = sm.cstart[cell];
-            const int nrec = lane_on ? sm.cend[cell] - c0 : 0;
-            if (BWD) {
-                if (nrec > 0) scatter_list<V>(go, on, sm.rec + c0, nrec, gfv);
-            } else {
-                const int maxn = __reduce_max_sync(FULL, nrec);
-                gather_list<V, BF16, kWide>(acc, sm.rec + c0, nrec, maxn, featv);
-            }
-            __syncwarp();
-        }
-        if (BWD) continue;
-
-        // ---- the one store of every output vector
-        if (lane_on) {
-            const int count = sm.cnt[cell];
-            const float gn = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-            float *o = p.out + ocell * p.C;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int vi = vec0 + v * vstep;
-                if (vi < p.vecs) {
-#pragma unroll
-                    for (int e = 0; e < PV; e += 2) {
-                        float4 *dst = reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2);
-                        float4 val = make_float4(acc[v][e].x * gn, acc[v][e].y * gn, acc[v][e + 1].x * gn, acc[v][e + 1].y * gn);
-                        if (p.accumulate) {  // multi-resolution levels after the first: `dst` holds the other levels' sum
-                            const float4 prev = *dst;
-                            val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
-                        }
-                        if (p.out_bf16) {
-                            uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C;
-                            *reinterpret_cast<uint2 *>(ob + (size_t)vi * (PV * 2) + e * 2) =
-                                make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
-                        } else {
-                            __stcs(dst, val);
+                    for (int v = 0; v < V; ++v) {
+                        const int vi = vec0 + v * vstep;
+                        go[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        on[v] = lane_on && vi < p.vecs;
+                        if (on[v] && cw_hi > cw_lo) {
+                            go[v] = __ldg(reinterpret_cast<const float4 *>(p.gout + ocell * p.C) + vi);
+                            go[v].x *= gscale, go[v].y *= gscale, go[v].z *= gscale, go[v].w *= gscale;
                         }
                     }
                 }
+
+                while (pos < sw_hi) {
+                    // a sub-block whose runs do not fit one round: its accumulators live across the walkers (rare)
+                    if (pos >= wb) wa = pos, wb = emit_round(p, cx, wa, nw);
+                    const int upto = min(sw_hi, wb);
+                    // this lane's cell: its runs inside [pos, upto)
+                    const int lw = min(max(cw_lo, pos), upto), hw = min(max(cw_hi, pos), upto);
+                    const int c0 = sm.woff[lw] - sm.woff[wa];
+                    const int nrec = (lane_on && !(p.dbg & 1)) ? sm.woff[hw] - sm.woff[lw] : 0;
+                    if (BWD) {
+                        if (nrec > 0) scatter_list<V>(go, on, sm.roff + c0, sm.rw + c0, nrec, p.rstep, gfv);
+                    } else {
+                        gather_list<V, BF16, kWide>(acc, sm.roff + c0, sm.rw + c0, nrec, p.rstep, featv);
+                    }
+                    pos = upto;
+                }
+                if (BWD) continue;
+
+                // ---- the one store of every output vector
+                if (lane_on) {
+                    const int count = sm.cnt[cell];
+                    const float gn = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
+                    float *o = p.out + ocell * p.C;
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        const int vi = vec0 + v * vstep;
+                        if (vi < p.vecs) {
+#pragma unroll
+                            for (int e = 0; e < PV; e += 2) {
+                                float4 *dst = reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2);
+                                float4 val = make_float4(acc[v][e].x * gn, acc[v][e].y * gn, acc[v][e + 1].x * gn, acc[v][e + 1].y * gn);
+                                if (p.accumulate) {  // multi-resolution levels after the first: `dst` holds the other levels' sum
+                                    const float4 prev = *dst;
+                                    val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
+                                }
+                                if (p.out_bf16) {
+                                    uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C;
+                                    *reinterpret_cast<uint2 *>(ob + (size_t)vi * (PV * 2) + e * 2) =
+                                        make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
+                                } else {
+                                    __stcs(dst, val);
+                                }
+                            }
+                        }
+                    }
+                    if (p.count_out && gl == 0 && blockIdx.y == 0) p.count_out[ocell] = count;
+                }
             }
-            if (p.count_out && gl == 0 && blockIdx.y == 0) p.count_out[ocell] = count;
+            s0 = s1;
         }
         __syncwarp();
     }

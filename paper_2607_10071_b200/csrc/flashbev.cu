@@ -54,7 +54,8 @@ struct KParams {
     float inv_n;                // 1 / N
     int blocks_x, blocks_y;     // super-blocks per batch element
     int band, reps;             // super-block order: bands of `band` rows; super-blocks per warp
-    int walk;                   // height bins per run (2 walk <= slots)
+    int walk, walk_shift;       // height bins (or texel rows) per run: a power of two, 2 walk <= slots
+    int inv_g;                  // ceil(65536 / g)
     int slots;                  // record slots per warp
     int colcap;                 // column descriptors per warp (>= cpw * N)
     int wcap;                   // runs per warp (= column descriptors per warp * ceil(Z / walk))
@@ -730,7 +731,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     k.rstep = p->feat_w > 1 ? k.vecs : 0;
     k.nvec_cam = p->N * p->feat_h * p->feat_w * k.vecs;  // < 2^31: tiled_applicable
     k.inv_n = 1.0f / (float)p->N;
-    k.dbg = (p->tune[3] >> 28) & 7;
+    k.dbg = (p->tune[3] >> 28) & 15;
 
     // channel mapping: V vectors per lane, g lanes per cell
     V = p->tune[0];
@@ -748,6 +749,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     warps = p->tune[3] & 0xf;
     if (!(warps == 1 || warps == 2 || warps == 4 || warps == 8)) warps = 4;
     k.g = g;
+    k.inv_g = (65536 + g - 1) / g;
     int cpw = std::min(32 / g, kMaxCpw);
     cpw = std::min(cpw, std::max(1, kColCapMax / p->N));  // a sub-block's candidate columns fit the descriptor table
     // sub-block of wx x wy cells, near-square, y (the contiguous output axis) the longer side
@@ -760,15 +762,17 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
 
     // record slots per warp and bins per run (a run writes at most two records per bin)
     const int slots_tune = (p->tune[3] >> 20) & 0xff;
-    k.slots = slots_tune ? std::max(64, slots_tune * 16) : 320;
+    k.slots = slots_tune ? std::max(64, slots_tune * 16) : 512;
     // a run is at most `walk` height bins, or `walk` texel rows of a column that moves at most two rows per bin
     const int units = std::max(p->Z, std::min(p->feat_h, 2 * p->Z + 2));  // per column at most
     k.walk = (p->tune[2] >= 1 && p->tune[2] <= 256) ? p->tune[2] : 16;
     k.walk = std::min(k.walk, std::min(units, (k.slots - 2) / 2));
     k.colcap = std::max(32, (k.cpw * p->N + 7) / 8 * 8);
+    for (k.walk_shift = 0; (2 << k.walk_shift) <= k.walk; ++k.walk_shift) {}
+    k.walk = 1 << k.walk_shift;
     int runs = (units + k.walk - 1) / k.walk;
-    while (k.colcap * runs > 2048 && k.walk < std::min(256, (k.slots - 2) / 2)) {  // keep the run table small: longer runs
-        k.walk = std::min(std::min(256, (k.slots - 2) / 2), k.walk * 2);
+    while (k.colcap * runs > 2048 && 2 * k.walk <= std::min(256, (k.slots - 2) / 2)) {  // keep the run table small: longer runs
+        k.walk *= 2, k.walk_shift += 1;
         runs = (units + k.walk - 1) / k.walk;
     }
 
@@ -783,13 +787,14 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     };
     if (sbx < 1 || sby < 1 || !fits(sbx, sby)) {
         static const int shapes[][2] = {{1, 1}, {1, 2}, {2, 2}, {2, 3}, {2, 4}, {3, 3}, {3, 4}, {4, 4}};
-        const int want = std::max(k.cpw, (int)(k.slots / (0.7 * std::min(p->Z, 2 * p->feat_h) + 8.0)));
+        // ... and few enough that every SM sees several waves of warps (a warp's latency is the kernel's)
+        const long long cells = (long long)p->B * p->X * p->Y;
+        const int want = (int)std::max<long long>(k.cpw, std::min<long long>((long long)(k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0)),
+                                                                          cells / ((long long)sm_count() * 60)));
         sbx = sby = 1;
         for (const auto &sh : shapes) {
             const int ct = sh[0] * sh[1] * k.cpw;
             if (!fits(sh[0], sh[1]) || ct > want) break;
-            // small problems: rather more warps than idle SMs (a warp's latency is the kernel's)
-            if (ct > k.cpw && (long long)p->B * p->X * p->Y / ct < (long long)sm_count() * 24) break;
             sbx = sh[0], sby = sh[1];
         }
     }
@@ -798,7 +803,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     k.ct = k.sbn * k.cpw;
     k.blocks_x = (p->X + sbx * k.wx - 1) / (sbx * k.wx);
     k.blocks_y = (p->Y + sby * k.wy - 1) / (sby * k.wy);
-    k.band = 4;
+    { const int bc = (p->tune[3] >> 18) & 3; k.band = bc == 1 ? 1 : (bc == 2 ? 2 : (bc == 3 ? 8 : 4)); }
     k.reps = (p->tune[3] >> 12) & 0xf;
     if (k.reps < 1) k.reps = 1;
     k.wcap = k.colcap * runs;

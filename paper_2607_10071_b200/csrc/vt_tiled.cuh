@@ -166,49 +166,75 @@ __device__ __forceinline__ void ldg_pair(const uint4 *ptr, uint4 &a, uint4 &b)
         : "l"(ptr));
 }
 
-// Gather of one cell list by its channel lanes, U records per iteration.  Every record is two taps of one
-// texel row, both always loadable.  The slots after a list hold loadable offsets too (another cell's records,
-// older ones, or zeros): the last iteration reads them and gives them weight 0.
+// base + 16 * index in one widening multiply-add
+__device__ __forceinline__ const uint4 *vec_at(const uint4 *base, unsigned index)
+{
+    const uint4 *r;
+    asm("mad.wide.u32 %0, %1, 16, %2;" : "=l"(r) : "r"(index), "l"(base));
+    return r;
+}
+
+// shared-memory loads through 32-bit shared-window addresses
+__device__ __forceinline__ unsigned lds_u32(unsigned addr)
+{
+    unsigned v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float2 lds_f32x2(unsigned addr)
+{
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
+}
+
+// U records of one cell list: two taps each, both always loadable; packed fp32 FMAs into the accumulators.
+template <int U, int V, bool BF16, bool WIDE>
+__device__ __forceinline__ void gather_records(float2 (&acc)[V][BF16 ? 4 : 2], unsigned loff, unsigned lw, unsigned rstep,
+                                               const uint4 *const (&featv)[V])
+{
+    unsigned ro[U];
+    float2 rw[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) ro[u] = lds_u32(loff + 4 * u), rw[u] = lds_f32x2(lw + 8 * u);
+    uint4 t[U][2][V];
+    if (WIDE) {  // the lane's vectors are adjacent: V / 2 loads of 32 bytes per tap
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int v = 0; v + 1 < V; v += 2) {
+                ldg_pair(vec_at(featv[v], ro[u]), t[u][0][v], t[u][0][v + 1]);
+                ldg_pair(vec_at(featv[v], ro[u] + rstep), t[u][1][v], t[u][1][v + 1]);
+            }
+    } else {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                t[u][0][v] = __ldg(vec_at(featv[v], ro[u]));
+                t[u][1][v] = __ldg(vec_at(featv[v], ro[u] + rstep));
+            }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            fma_vec<BF16>(acc[v], t[u][0][v], make_float2(rw[u].x, rw[u].x));
+            fma_vec<BF16>(acc[v], t[u][1][v], make_float2(rw[u].y, rw[u].y));
+        }
+}
+
+// Gather of one cell list by its channel lanes: groups of U records, then the rest one by one.
+// loff / lw: shared-window addresses of the list's offsets and weights.
 template <int V, bool BF16, bool WIDE>
-__device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], const int *loff, const float2 *lw, int nrec, int rstep,
+__device__ __forceinline__ void gather_list(float2 (&acc)[V][BF16 ? 4 : 2], unsigned loff, unsigned lw, int nrec, unsigned rstep,
                                             const uint4 *const (&featv)[V])
 {
     constexpr int U = V == 1 ? 4 : (V == 2 ? (BF16 ? FB_U_BF16V2 : 2) : 1);
-    for (int j = 0; j < nrec; j += U) {
-        int ro[U];
-        float2 rw[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) ro[u] = loff[j + u], rw[u] = lw[j + u];
-        uint4 t[U][2][V];
-        if (WIDE) {  // the lane's vectors are adjacent: V / 2 loads of 32 bytes per tap
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int v = 0; v + 1 < V; v += 2) {
-                    ldg_pair(featv[v] + ro[u], t[u][0][v], t[u][0][v + 1]);
-                    ldg_pair(featv[v] + ro[u] + rstep, t[u][1][v], t[u][1][v + 1]);
-                }
-        } else {
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    t[u][0][v] = __ldg(featv[v] + ro[u]);
-                    t[u][1][v] = __ldg(featv[v] + ro[u] + rstep);
-                }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const bool has = j + u < nrec;
-            const float wl = has ? rw[u].x : 0.f;
-            const float wr = has ? rw[u].y : 0.f;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                fma_vec<BF16>(acc[v], t[u][0][v], make_float2(wl, wl));
-                fma_vec<BF16>(acc[v], t[u][1][v], make_float2(wr, wr));
-            }
-        }
-    }
+    int j = 0;
+    for (; j + U <= nrec; j += U, loff += 4 * U, lw += 8 * U) gather_records<U, V, BF16, WIDE>(acc, loff, lw, rstep, featv);
+    if (U > 1)
+        for (; j < nrec; ++j, loff += 4, lw += 8) gather_records<1, V, BF16, WIDE>(acc, loff, lw, rstep, featv);
 }
 
 // Backward of the gather: every record adds its two weighted taps of the cell's output gradient to the
@@ -269,9 +295,10 @@ __device__ __forceinline__ int column_build(const KParams &p, const double *mats
     float lo = -1.f, hi = (float)p.Z;
     bool empty = false;
     auto cond = [&](float a, float bslope) {
-        if (bslope > 0.f) lo = fmaxf(lo, -a * __frcp_rn(bslope));       // k > -a/b
-        else if (bslope < 0.f) hi = fminf(hi, -a * __frcp_rn(bslope));  // k < -a/b
-        else if (a <= 0.f) empty = true;  // independent of z (NaN: keep, tested exactly below)
+        const float t = -a * __frcp_rn(bslope);                  // the condition changes sign at k = t
+        lo = bslope > 0.f ? fmaxf(lo, t) : lo;                   // k > -a/b
+        hi = bslope < 0.f ? fminf(hi, t) : hi;                   // k < -a/b
+        empty |= (bslope == 0.f) & (a <= 0.f);                   // independent of z (NaN: keep, tested exactly below)
     };
     const double d0 = fma(m[10], zc0, a2);
     const double p00 = fma(m[2], zc0, a0);
@@ -339,17 +366,12 @@ __device__ __forceinline__ int affine_units(const KParams &p, const ColDesc &D, 
 }
 
 // Records of a run of an affine column: [u0, u0 + len) are rows counted from the column's first written row, or bins.
-__device__ __forceinline__ int affine_run_records(const KParams &p, const ColDesc &D, int u0, int len)
-{
-    if (affine_by_rows(D)) return len;
-    const int r_first = (int)floor(fma((double)u0, D.d1, D.d0)), r_last = (int)floor(fma((double)(u0 + len - 1), D.d1, D.d0));
-    return 2 * len - (r_first < 0 ? 1 : 0) - (r_last + 1 > p.Hf - 1 ? 1 : 0);
-}
+__device__ __forceinline__ int affine_run_records(const ColDesc &D, int len) { return affine_by_rows(D) ? len : 2 * len; }
 
 // ---- step 2: walker of an affine column.  Writes exactly affine_run_records() records. -------------------------
 // A run of rows [ra, rb) takes the bins whose upper tap lies in rows ra - 1 .. rb - 1: a row's weight is the (1 - ty)
 // of the bins in it plus the ty of the bins in the row above, so every run is complete by itself and neighbouring
-// runs share no record.
+// runs share no record.  The run's own record slots serve as the accumulators of its rows.
 __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm, const ColDesc &D, int u0, int len,
                                             int *out_off, float2 *out_w, int cap)
 {
@@ -368,12 +390,10 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
     const int dstep = rev ? -1 : 1;
     const int rowv = p.Wf * p.vecs, offc = D.f.offc;
     const double S = D.d1, A = D.d0;
-    const bool by_rows = affine_by_rows(D);
 
-    int kb = u0, ke = u0 + len;  // bins [kb, ke)
-    int ra = 0, rb = p.Hf;       // rows written: [ra, rb)
-    if (by_rows) {
-        ra = max((int)floor(A), 0) + u0, rb = ra + len;
+    if (affine_by_rows(D)) {
+        len = min(len, cap);  // (never cuts: the run's slots were counted from the same numbers)
+        const int ra = max((int)floor(A), 0) + u0;
         const double inv = (double)__frcp_rn((float)S);
         auto first_bin_at = [&](double rr) {  // smallest k' in [0, nb] with A + k' S >= rr
             double e = ceil((rr - A) * inv);
@@ -383,52 +403,50 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
             else if (k < nb && fma((double)k, S, A) < rr) ++k;
             return k;
         };
-        kb = first_bin_at((double)(ra - 1)), ke = first_bin_at((double)rb);
-    }
-    int n = 0;
-    auto emit = [&](int row, float w) {
-        if (row >= ra && row < rb) {
-            const int at = by_rows ? row - ra : n;
-            if (at < cap) {
-                out_off[at] = FB_IDX(offc + row * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
-                out_w[at] = make_float2(cl * w, cr * w);
+        const int kb = first_bin_at((double)(ra - 1)), ke = first_bin_at((double)(ra + len));
+        float *w = reinterpret_cast<float *>(out_w);  // w[2 i]: weight of row ra + i
+        for (int i = 0; i < len; ++i) w[2 * i] = 0.f;
+        double kd = (double)kb;
+        const unsigned char *dk = den + kb * dstep;
+        for (int k = kb; k < ke; ++k, kd += 1.0, dk += dstep) {
+            const double fy = fma(kd, S, A), fl = floor(fy);
+            const int i = (int)fl - ra;  // row of the upper tap, relative
+            float ty = (float)(fy - fl), tu = 1.f - ty;
+            if (eq1) {
+                const float sc = 1.f / (float)max(1, (int)*dk);
+                ty *= sc, tu *= sc;
             }
-            ++n;
+            if ((unsigned)i < (unsigned)len) w[2 * i] += tu;
+            if ((unsigned)(i + 1) < (unsigned)len) w[2 * i + 2] += ty;
         }
-    };
-    if (kb >= ke) {  // (cannot happen: a run of rows always has bins, a run of bins has len >= 1; leave no stale weights)
-        for (int i = 0; i < min(len, cap); ++i) out_off[i] = offc, out_w[i] = make_float2(0.f, 0.f);
-        return;
-    }
-    double kd = (double)kb;
-    int ro;
-    float wu, wl;
-    {
-        const double fy = fma(kd, S, A), fl = floor(fy);
-        const float ty = (float)(fy - fl);
-        const float s = eq1 ? 1.f / (float)max(1, (int)den[kb * dstep]) : 1.f;
-        ro = (int)fl;
-        wu = (1.f - ty) * s, wl = ty * s;
-    }
-    for (int k = kb + 1; k < ke; ++k) {
-        kd += 1.0;
-        const double fy = fma(kd, S, A), fl = floor(fy);
-        const int r = (int)fl;
-        const float ty = (float)(fy - fl);
-        const float s = eq1 ? 1.f / (float)max(1, (int)den[k * dstep]) : 1.f;
-        if (r != ro) {
-            emit(ro, wu);
-            if (!by_rows || r != ro + 1) {
-                emit(ro + 1, wl);
-                wl = 0.f;
+        int off = FB_IDX(offc + ra * rowv, p.nvec_cam - p.vecs - p.rstep + 1 - (len - 1) * rowv, p.err);
+        for (int i = 0; i < len; ++i, off += rowv) {
+            const float wi = w[2 * i];
+            out_w[i] = make_float2(cl * wi, cr * wi);
+            out_off[i] = off;
+        }
+    } else {
+        // rows of successive bins never coincide: two records per bin (a row outside the map: weight 0, clamped)
+        len = min(len, cap / 2);
+        double kd = (double)u0;
+        const unsigned char *dk = den + u0 * dstep;
+        for (int i = 0; i < len; ++i, kd += 1.0, dk += dstep) {
+            const double fy = fma(kd, S, A), fl = floor(fy);
+            const int r = (int)fl;
+            float ty = (float)(fy - fl), tu = 1.f - ty;
+            if (eq1) {
+                const float sc = 1.f / (float)max(1, (int)*dk);
+                ty *= sc, tu *= sc;
             }
-            wu = wl, wl = 0.f, ro = r;
+            if (r < 0) tu = 0.f;
+            if (r + 1 > p.Hf - 1) ty = 0.f;
+            const int ru = max(r, 0), rl = min(r + 1, p.Hf - 1);
+            out_off[2 * i] = FB_IDX(offc + ru * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
+            out_w[2 * i] = make_float2(cl * tu, cr * tu);
+            out_off[2 * i + 1] = FB_IDX(offc + rl * rowv, p.nvec_cam - p.vecs - p.rstep + 1, p.err);
+            out_w[2 * i + 1] = make_float2(cl * ty, cr * ty);
         }
-        wu = fmaf(1.f - ty, s, wu);
-        wl = fmaf(ty, s, wl);
     }
-    emit(ro, wu);
-    emit(ro + 1, wl);
 }
 
 // ---- step 2: walker of a general column (every bin projected in fp64).  COUNT-only or EMIT. ------------------------
@@ -570,7 +588,7 @@ __device__ __forceinline__ int build_columns(const KParams &p, WarpCtx cx, int j
             affine = (D.meta >> 12) & 1;
             if (affine) units = affine_units(p, D, nb, row_first);
         }
-        const int runs = (units + p.walk - 1) / p.walk;
+        const int runs = (units + p.walk - 1) >> p.walk_shift;  // walk is a power of two
         int x = runs;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -586,7 +604,7 @@ __device__ __forceinline__ int build_columns(const KParams &p, WarpCtx cx, int j
                 const int u0 = i * p.walk, len = min(p.walk, units - u0);
                 sm.wk[FB_IDX(wbase + i, p.wcap, p.err)] = (uint32_t)j | ((uint32_t)u0 << 8) | ((uint32_t)(len - 1) << 24);
                 sm.woff[FB_IDX(wbase + i, p.wcap + 1, p.err)] = mine;
-                mine += affine ? affine_run_records(p, D, u0, len) : walk_general<false>(p, sm, cx.mats, D, u0, len, nullptr, nullptr, 0);
+                mine += affine ? affine_run_records(D, len) : walk_general<false>(p, sm, cx.mats, D, u0, len, nullptr, nullptr, 0);
             }
         }
         int y = mine;
@@ -708,11 +726,12 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
         celltab[c] = v;
     }
     // every record slot always holds loadable offsets: the gather may read (not use) slots past a list
-    for (int i = lane; i < p.slots + 4; i += 32) sm.roff[i] = 0, sm.rw[i] = make_float2(0.f, 0.f);
+    for (int i = lane; i < (p.slots + 4) / 4; i += 32) reinterpret_cast<int4 *>(sm.roff)[i] = make_int4(0, 0, 0, 0);
+    for (int i = lane; i < (p.slots + 4) / 2; i += 32) reinterpret_cast<float4 *>(sm.rw)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();  // the only CTA-wide barrier
 
     // ---- gather role of this lane inside a sub-block
-    const int cg = lane / p.g, gl = lane - cg * p.g;
+    const int cg = (lane * p.inv_g) >> 16, gl = lane - cg * p.g;  // lane / g
     const bool role = cg < p.cpw;
     constexpr bool kWide = WIDE && V >= 2 && !BWD;
     const int vstep = kWide ? 1 : p.g;  // distance between the lane's channel vectors
@@ -730,6 +749,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
         }
     }
     const int my_tab = celltab[lane];
+    const unsigned roff_s = (unsigned)__cvta_generic_to_shared(sm.roff), rw_s = (unsigned)__cvta_generic_to_shared(sm.rw);
 
     for (int rep = 0; rep < p.reps; ++rep) {
         // ---- which super-block: ids run along y inside bands of `band` rows of super-blocks
@@ -751,7 +771,13 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
             in_mask = __ballot_sync(FULL, in);
         }
         __syncwarp();
-        survey_candidates(p, cx, in_mask);
+        if (p.dbg & 8) {
+            sm.cfirst[lane] = 0;
+            if (lane == 0) sm.cfirst[32] = 0;
+            __syncwarp();
+        } else {
+            survey_candidates(p, cx, in_mask);
+        }
 
         // ---- segments: as many sub-blocks as have at most `colcap` surviving columns together (normally all of them)
         for (int s0 = 0; s0 < p.sbn;) {
@@ -809,7 +835,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                     if (BWD) {
                         if (nrec > 0) scatter_list<V>(go, on, sm.roff + c0, sm.rw + c0, nrec, p.rstep, gfv);
                     } else {
-                        gather_list<V, BF16, kWide>(acc, sm.roff + c0, sm.rw + c0, nrec, p.rstep, featv);
+                        gather_list<V, BF16, kWide>(acc, roff_s + 4 * c0, rw_s + 8 * c0, nrec, (unsigned)p.rstep, featv);
                     }
                     pos = upto;
                 }

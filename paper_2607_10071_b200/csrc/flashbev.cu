@@ -766,12 +766,13 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     // a run is at most `walk` height bins, or `walk` texel rows of a column that moves at most two rows per bin
     const int units = std::max(p->Z, std::min(p->feat_h, 2 * p->Z + 2));  // per column at most
     k.walk = (p->tune[2] >= 1 && p->tune[2] <= 256) ? p->tune[2] : 16;
-    k.walk = std::min(k.walk, std::min(units, (k.slots - 2) / 2));
+    // (the rounds of a sub-block whose records exceed the slots need 2 walk (cells + 1) <= slots)
+    k.walk = std::max(1, std::min(k.walk, std::min(units, k.slots / (2 * (k.cpw + 1)))));
     k.colcap = std::max(32, (k.cpw * p->N + 7) / 8 * 8);
     for (k.walk_shift = 0; (2 << k.walk_shift) <= k.walk; ++k.walk_shift) {}
     k.walk = 1 << k.walk_shift;
     int runs = (units + k.walk - 1) / k.walk;
-    while (k.colcap * runs > 2048 && 2 * k.walk <= std::min(256, (k.slots - 2) / 2)) {  // keep the run table small: longer runs
+    while (k.colcap * runs > 2048 && 2 * k.walk <= std::min(256, k.slots / (2 * (k.cpw + 1)))) {  // keep the run table small: longer runs
         k.walk *= 2, k.walk_shift += 1;
         runs = (units + k.walk - 1) / k.walk;
     }

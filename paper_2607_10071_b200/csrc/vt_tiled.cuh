@@ -645,33 +645,14 @@ __device__ __forceinline__ int build_columns(const KParams &p, WarpCtx cx, int j
     return nw;
 }
 
-// ---- step 2: a round.  As many runs from `wa` on as fit the record slots are walked, one lane each; returns the
-// first run not taken.
-__device__ FB_EMIT_INLINE int emit_round(const KParams &p, WarpCtx cx, int wa, int nw)
+// ---- step 2: run w is walked by the calling lane; its records go to slots [at, at + its count) ------------------
+__device__ __forceinline__ void walk_one(const KParams &p, const WarpSmem &sm, const double *mats, int w, int at)
 {
-    constexpr unsigned FULL = 0xffffffffu;
-    const WarpSmem sm = warp_smem(p, cx.warp_base);
-    const int lane = threadIdx.x & 31;
-    __syncwarp();
-    const int base = sm.woff[wa];
-    int wb = wa;
-    for (int w0 = wa + 1; w0 <= nw; w0 += 32) {
-        const int w = w0 + lane;
-        const bool fits = w <= nw && sm.woff[w] - base <= p.slots;
-        const unsigned bal = __ballot_sync(FULL, fits);
-        wb = w0 - 1 + __popc(bal);
-        if (bal != FULL) break;
-    }
-    if (wb <= wa) wb = wa + 1;  // (cannot happen: one run always fits; never loop without progress)
-    for (int w = wa + lane; w < wb && !(p.dbg & 2); w += 32) {
-        const uint32_t wd = sm.wk[w];
-        const ColDesc D = sm.col[FB_IDX(wd & 0xff, p.colcap, p.err)];
-        const int at = FB_IDX(sm.woff[w] - base, p.slots, p.err);
-        if ((D.meta >> 12) & 1) walk_affine(p, sm, D, (wd >> 8) & 0xffff, (wd >> 24) + 1, sm.roff + at, sm.rw + at, p.slots - at);
-        else walk_general<true>(p, sm, cx.mats, D, (wd >> 8) & 0xffff, (wd >> 24) + 1, sm.roff + at, sm.rw + at, p.slots - at);
-    }
-    __syncwarp();
-    return wb;
+    const uint32_t wd = sm.wk[w];
+    const ColDesc D = sm.col[FB_IDX(wd & 0xff, p.colcap, p.err)];
+    at = FB_IDX(at, p.slots, p.err);
+    if ((D.meta >> 12) & 1) walk_affine(p, sm, D, (wd >> 8) & 0xffff, (wd >> 24) + 1, sm.roff + at, sm.rw + at, p.slots - at);
+    else walk_general<true>(p, sm, mats, D, (wd >> 8) & 0xffff, (wd >> 24) + 1, sm.roff + at, sm.rw + at, p.slots - at);
 }
 
 // WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
@@ -787,8 +768,9 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
             const int ncols = sm.cfirst[min(s1 * p.cpw, p.ct)] - jb;  // <= colcap: a sub-block has at most cpw * N candidates
             const int nw = (p.dbg & 4) ? 0 : build_columns(p, cx, jb, ncols, s0 * p.cpw, min(s1 * p.cpw, p.ct));
 
-            // ---- rounds of runs [wa, wb) that fit the record slots; gather sub-block by sub-block
-            int wa = 0, wb = 0;
+            // ---- rounds: the runs of as many whole sub-blocks as fit the record slots are walked together (one lane
+            // per run), then the sub-blocks are gathered one by one
+            int wa = 0, wb = 0;  // the current round holds runs [wa, wb)
             for (int s = s0; s < s1; ++s) {
                 const int cell = s * p.cpw + (role ? cg : 0);
                 const bool lane_on = role && ((in_mask >> cell) & 1u);
@@ -799,8 +781,20 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                 int sw_lo = sm.colw[sm.cfirst[s * p.cpw] - jb], sw_hi = sm.colw[sm.cfirst[min((s + 1) * p.cpw, p.ct)] - jb];
                 int cw_lo = sm.colw[sm.cfirst[cell] - jb], cw_hi = sm.colw[sm.cfirst[cell + 1] - jb];  // this lane's cell
                 if (p.dbg & 4) sw_lo = sw_hi = cw_lo = cw_hi = 0;
-                int pos = sw_lo;  // runs of this sub-block before `pos` are done
-                if (pos < sw_hi && pos >= wb) wa = pos, wb = emit_round(p, cx, wa, nw);  // (no accumulator is live here)
+                const int sub_records = sm.woff[sw_hi] - sm.woff[sw_lo];
+                const bool oversized = sub_records > p.slots;
+                if (!oversized && sw_hi > wb) {
+                    __syncwarp();
+                    wa = sw_lo, wb = sw_hi;
+                    for (int s2 = s + 1; s2 < s1; ++s2) {
+                        const int hi2 = sm.colw[sm.cfirst[min((s2 + 1) * p.cpw, p.ct)] - jb];
+                        if (sm.woff[hi2] - sm.woff[wa] > p.slots) break;
+                        wb = hi2;
+                    }
+                    const int base = sm.woff[wa];
+                    for (int w = wa + lane; w < wb && !(p.dbg & 2); w += 32) walk_one(p, sm, mats, w, sm.woff[w] - base);
+                    __syncwarp();
+                }
 
                 float2 acc[V][PV];
 #pragma unroll
@@ -824,20 +818,44 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                     }
                 }
 
-                while (pos < sw_hi) {
-                    // a sub-block whose runs do not fit one round: its accumulators live across the walkers (rare)
-                    if (pos >= wb) wa = pos, wb = emit_round(p, cx, wa, nw);
-                    const int upto = min(sw_hi, wb);
-                    // this lane's cell: its runs inside [pos, upto)
-                    const int lw = min(max(cw_lo, pos), upto), hw = min(max(cw_hi, pos), upto);
-                    const int c0 = sm.woff[lw] - sm.woff[wa];
-                    const int nrec = (lane_on && !(p.dbg & 1)) ? sm.woff[hw] - sm.woff[lw] : 0;
+                if (!oversized) {
+                    const int c0 = sm.woff[cw_lo] - sm.woff[wa];
+                    const int nrec = (lane_on && !(p.dbg & 1)) ? sm.woff[cw_hi] - sm.woff[cw_lo] : 0;
                     if (BWD) {
                         if (nrec > 0) scatter_list<V>(go, on, sm.roff + c0, sm.rw + c0, nrec, p.rstep, gfv);
                     } else {
                         gather_list<V, BF16, kWide>(acc, roff_s + 4 * c0, rw_s + 8 * c0, nrec, (unsigned)p.rstep, featv);
                     }
-                    pos = upto;
+                } else {
+                    // A sub-block whose records exceed the slots: several rounds of as many runs as fit, in order; the
+                    // accumulators live across the walkers here.
+                    int pos = sw_lo;
+                    while (pos < sw_hi) {
+                        __syncwarp();
+                        const int base = sm.woff[pos];
+                        int upto = pos;
+                        for (int w0 = pos + 1; w0 <= sw_hi; w0 += 32) {
+                            const int w = w0 + lane;
+                            const bool fits = w <= sw_hi && sm.woff[w] - base <= p.slots;
+                            const unsigned bal = __ballot_sync(FULL, fits);
+                            upto = w0 - 1 + __popc(bal);
+                            if (bal != FULL) break;
+                        }
+                        if (upto <= pos) upto = pos + 1;  // (cannot happen: one run always fits; never loop without progress)
+                        for (int w = pos + lane; w < upto && !(p.dbg & 2); w += 32) walk_one(p, sm, mats, w, sm.woff[w] - base);
+                        __syncwarp();
+                        // this lane's cell: its runs inside [pos, upto)
+                        const int lw = min(max(cw_lo, pos), upto), hw = min(max(cw_hi, pos), upto);
+                        const int c0 = sm.woff[lw] - base;
+                        const int nrec = (lane_on && !(p.dbg & 1)) ? sm.woff[hw] - sm.woff[lw] : 0;
+                        if (BWD) {
+                            if (nrec > 0) scatter_list<V>(go, on, sm.roff + c0, sm.rw + c0, nrec, p.rstep, gfv);
+                        } else {
+                            gather_list<V, BF16, kWide>(acc, roff_s + 4 * c0, rw_s + 8 * c0, nrec, (unsigned)p.rstep, featv);
+                        }
+                        pos = upto;
+                    }
+                    wa = wb = sw_hi;
                 }
                 if (BWD) continue;
 

@@ -738,12 +738,12 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     int g = p->tune[1];
     if (!(V == 1 || V == 2 || V == 4) || g < 1 || g > 32) V = 0, g = 0;
     if (!V) {
-        // tall columns: eight cells per sub-block
+        // (measured) up to 8 vectors per texel: one per lane; up to 32: two adjacent ones per lane; beyond: four.
+        // Tall columns of 8-vector texels: eight cells per sub-block amortise the geometry better.
         if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
         else if (k.vecs <= 8) V = 1, g = k.vecs;
-        else if (k.vecs <= 16) V = (k.vecs % 2 == 0) ? 2 : 1, g = (k.vecs + V - 1) / V;
-        else if (k.vecs < 24 || (k.vecs <= 32 && p->Z >= 16)) V = 2, g = (k.vecs + 1) / 2;
-        else V = 4, g = (k.vecs + 3) / 4;  // wide texels: four vectors per lane keep 2-5 cells in a sub-block
+        else if (k.vecs <= 32) V = (k.vecs % 2 == 0 || k.vecs > 16) ? 2 : 1, g = (k.vecs + V - 1) / V;
+        else V = 4, g = (k.vecs + 3) / 4;
         if (g > 32) g = 32;
     }
     warps = p->tune[3] & 0xf;
@@ -788,10 +788,10 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     };
     if (sbx < 1 || sby < 1 || !fits(sbx, sby)) {
         static const int shapes[][2] = {{1, 1}, {1, 2}, {2, 2}, {2, 3}, {2, 4}, {3, 3}, {3, 4}, {4, 4}};
-        // ... and few enough that every SM sees several waves of warps (a warp's latency is the kernel's)
+        // ... at most four sub-blocks, and few enough cells that every SM still gets a full set of warps
         const long long cells = (long long)p->B * p->X * p->Y;
-        const int want = (int)std::max<long long>(k.cpw, std::min<long long>((long long)(k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0)),
-                                                                          cells / ((long long)sm_count() * 60)));
+        const int want = (int)std::max<long long>(k.cpw, std::min<long long>(std::min<long long>(4 * k.cpw, (long long)(k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0))),
+                                                                          cells / ((long long)sm_count() * 20)));
         sbx = sby = 1;
         for (const auto &sh : shapes) {
             const int ct = sh[0] * sh[1] * k.cpw;

@@ -34,8 +34,8 @@
 //          float  slope[N][5]   d/dk of the five validity conditions
 //          int    camfast[N]    1: the camera's depth and horizontal texel coordinate do not depend on height
 //          int    celltab[32]   position of cell c inside a super-block: lx | ly << 8
-//   warp : int     roff[slots + 4] row records of the current round: vector index of the first tap (the second follows
-//          float2  rw[slots + 4]   `rstep` vectors later) and the two weights (+ slack that is read, never used)
+//   warp : int     roff[slots]     row records of the current round: vector index of the first tap (the second follows
+//          float2  rw[slots]       `rstep` vectors later) and the two weights
 //          ColDesc col[ccap]       columns of the current segment, (cell, camera) order
 //          uint32  wk[wcap]        runs: column | first bin << 8 | (bins - 1) << 24
 //          int     woff[wcap + 1]  records before run w
@@ -101,8 +101,8 @@ __host__ __device__ inline size_t warp_smem_layout(unsigned char *base, WarpSmem
         o += align16(bytes);
         return ptr;
     };
-    unsigned char *p0 = take((size_t)(slots + 4) * sizeof(float2));
-    unsigned char *p0b = take((size_t)(slots + 4) * sizeof(int));
+    unsigned char *p0 = take((size_t)slots * sizeof(float2));
+    unsigned char *p0b = take((size_t)slots * sizeof(int));
     unsigned char *p1 = take((size_t)colcap * sizeof(ColDesc));
     unsigned char *p2 = take((size_t)ct * sizeof(double2));
     unsigned char *p3 = take((size_t)wcap * sizeof(uint32_t));
@@ -291,6 +291,41 @@ __device__ __forceinline__ int column_build(const KParams &p, const double *mats
     D.d0 = a0, D.d1 = a1, D.d2 = a2;
     D.kk = 1;  // klo = 1 > khi = 0: no bins
     D.meta = c | (n << 6);
+    if (camfast[n]) {
+        // Depth and fx do not depend on the height: one texel column, fy = ay + k sy affine in the bin index k, and
+        // the valid bins are those with -1/2 < fy < Hf - 1/2: an interval in closed form, its ends confirmed.
+        if (!(a2 > kDepthMin)) return 0;
+        const double r = fast_rcp(a2);
+        const double fx = fma(a0, r, -0.5);
+        const double wl = (double)p.Wf - 0.5, hl = (double)p.Hf - 0.5;
+        if (!(fx > -0.5 && fx < wl)) return 0;
+        const double ay = fma(fma(m[6], zc0, a1), r, -0.5), sy = m[6] * p.dz * r;
+        const double inv = fast_rcp(sy);
+        const double ta = (-0.5 - ay) * inv, tb = (hl - ay) * inv;      // fy crosses the two borders at these k
+        const double zf = (double)p.Z;
+        double tlo = sy > 0.0 ? ta : (sy < 0.0 ? tb : -1.0), thi = sy > 0.0 ? tb : (sy < 0.0 ? ta : zf);
+        tlo = fmin(fmax(tlo, -1.0), zf), thi = fmin(fmax(thi, -1.0), zf);  // NaN -> the whole range: every bin is then tested
+        int klo = max((int)floor(tlo), 0), khi = min((int)ceil(thi), p.Z - 1);
+        auto inside = [&](int k) {
+            const double fy = fma((double)k, sy, ay);
+            return (fy > -0.5) & (fy < hl);
+        };
+        while (klo <= khi && !inside(klo)) ++klo;
+        while (khi > klo && !inside(khi)) --khi;
+        if (klo > khi) return 0;
+        const bool rev = sy < 0.0;  // rows ascend with the renumbered bins k' = khi - k
+        const double flx = floor(fx);
+        const int x0 = (int)flx;
+        const int edge = x0 < 0 ? 1 : (x0 >= p.Wf - 1 ? 2 : 0);
+        const int xc = edge == 1 ? 0 : (edge == 2 ? max(p.Wf - 2, 0) : x0);
+        D.d0 = fma((double)(rev ? khi : klo), sy, ay);
+        D.d1 = rev ? -sy : sy;
+        D.f.offc = (n * p.Hf * p.Wf + xc) * p.vecs;
+        D.f.tx = (float)(fx - flx);
+        D.kk = klo | (khi << 16);
+        D.meta |= (1 << 12) | ((rev ? 1 : 0) << 13) | (edge << 14);
+        return khi - klo + 1;
+    }
     // conditions alpha + beta * k > 0 (k real): depth, left, right, top, bottom -> conservative interval
     float lo = -1.f, hi = (float)p.Z;
     bool empty = false;
@@ -333,21 +368,6 @@ __device__ __forceinline__ int column_build(const KParams &p, const double *mats
     const bool rev = khi > klo && fy_at < fy_lo;  // rows ascend with the renumbered bins k' = khi - k
     D.kk = klo | (khi << 16);
     D.meta |= (rev ? 1 : 0) << 13;
-    if (camfast[n]) {
-        // depth and fx do not depend on the height: one texel column, fy affine in the bin index
-        const double r = fast_rcp(a2);
-        const double fx = fma(a0, r, -0.5);
-        const double flx = floor(fx);
-        const int x0 = (int)flx;
-        const int edge = x0 < 0 ? 1 : (x0 >= p.Wf - 1 ? 2 : 0);
-        const int xc = edge == 1 ? 0 : (edge == 2 ? max(p.Wf - 2, 0) : x0);
-        const double sy = m[6] * p.dz * r;                 // fy step per bin
-        D.d0 = fma((double)(rev ? khi : klo), sy, fma(p10, r, -0.5));
-        D.d1 = rev ? -sy : sy;
-        D.f.offc = (n * p.Hf * p.Wf + xc) * p.vecs;
-        D.f.tx = (float)(fx - flx);
-        D.meta |= (1 << 12) | (edge << 14);
-    }
     return khi - klo + 1;
 }
 
@@ -706,9 +726,6 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
         }
         celltab[c] = v;
     }
-    // every record slot always holds loadable offsets: the gather may read (not use) slots past a list
-    for (int i = lane; i < (p.slots + 4) / 4; i += 32) reinterpret_cast<int4 *>(sm.roff)[i] = make_int4(0, 0, 0, 0);
-    for (int i = lane; i < (p.slots + 4) / 2; i += 32) reinterpret_cast<float4 *>(sm.rw)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();  // the only CTA-wide barrier
 
     // ---- gather role of this lane inside a sub-block
@@ -729,6 +746,10 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
             gfv[v] = BWD ? reinterpret_cast<float4 *>(p.gfeat) + cam0 + vi : nullptr;
         }
     }
+    const int out_lane = vec0 * (PV * 2), vstride = vstep * (PV * 2);  // channel of the lane's first vector; channels between its vectors
+    bool von[V];                                                         // the lane's v-th vector exists (ragged last channel block)
+#pragma unroll
+    for (int v = 0; v < V; ++v) von[v] = vec0 + v * vstep < p.vecs;
     const int my_tab = celltab[lane];
     const unsigned roff_s = (unsigned)__cvta_generic_to_shared(sm.roff), rw_s = (unsigned)__cvta_generic_to_shared(sm.rw);
 
@@ -862,29 +883,44 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                 // ---- the one store of every output vector
                 if (lane_on) {
                     const int count = sm.cnt[cell];
-                    const float gn = (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
-                    float *o = p.out + ocell * p.C;
+                    if (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) {
+                        const float gn = 1.f / (float)(count > 1 ? count : 1);
 #pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        const int vi = vec0 + v * vstep;
-                        if (vi < p.vecs) {
+                        for (int v = 0; v < V; ++v)
 #pragma unroll
-                            for (int e = 0; e < PV; e += 2) {
-                                float4 *dst = reinterpret_cast<float4 *>(o + (size_t)vi * (PV * 2) + e * 2);
-                                float4 val = make_float4(acc[v][e].x * gn, acc[v][e].y * gn, acc[v][e + 1].x * gn, acc[v][e + 1].y * gn);
-                                if (p.accumulate) {  // multi-resolution levels after the first: `dst` holds the other levels' sum
-                                    const float4 prev = *dst;
-                                    val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
-                                }
-                                if (p.out_bf16) {
-                                    uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C;
-                                    *reinterpret_cast<uint2 *>(ob + (size_t)vi * (PV * 2) + e * 2) =
-                                        make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
-                                } else {
-                                    __stcs(dst, val);
+                            for (int e = 0; e < PV; ++e) acc[v][e].x *= gn, acc[v][e].y *= gn;
+                    }
+                    float *o = p.out + ocell * p.C + out_lane;  // this lane's first channel of the cell
+                    if (!(p.accumulate | p.out_bf16)) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (von[v]) {
+#pragma unroll
+                                for (int e = 0; e < PV; e += 2)
+                                    __stcs(reinterpret_cast<float4 *>(o + v * vstride + e * 2),
+                                           make_float4(acc[v][e].x, acc[v][e].y, acc[v][e + 1].x, acc[v][e + 1].y));
+                            }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (von[v]) {
+#pragma unroll
+                                for (int e = 0; e < PV; e += 2) {
+                                    float4 *dst = reinterpret_cast<float4 *>(o + v * vstride + e * 2);
+                                    float4 val = make_float4(acc[v][e].x, acc[v][e].y, acc[v][e + 1].x, acc[v][e + 1].y);
+                                    if (p.accumulate) {  // multi-resolution levels after the first: `dst` holds the other levels' sum
+                                        const float4 prev = *dst;
+                                        val.x += prev.x, val.y += prev.y, val.z += prev.z, val.w += prev.w;
+                                    }
+                                    if (p.out_bf16) {
+                                        uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + ocell * p.C + out_lane;
+                                        *reinterpret_cast<uint2 *>(ob + v * vstride + e * 2) =
+                                            make_uint2(pack_bf16x2(val.x, val.y), pack_bf16x2(val.z, val.w));
+                                    } else {
+                                        __stcs(dst, val);
+                                    }
                                 }
                             }
-                        }
                     }
                     if (p.count_out && gl == 0 && blockIdx.y == 0) p.count_out[ocell] = count;
                 }

@@ -10,7 +10,9 @@
  * DEVICE pointer unless the entry point says otherwise.  The caller owns every
  * buffer.  Unless an entry point says otherwise the library allocates nothing,
  * frees nothing, keeps no pointer after return, never synchronises the device,
- * and enqueues its work on the caller's stream.  It is re-entrant and thread safe.
+ * and enqueues its work on the caller's stream.  It is re-entrant and thread safe; the only state it
+ * keeps is per host thread (what flashbev_last_launch_count / flashbev_last_kernel_name report) and a
+ * per-device cache of the multiprocessor count.
  */
 #ifndef FLASHBEV_H_
 #define FLASHBEV_H_
@@ -30,7 +32,9 @@ typedef enum flashbev_status {
     FLASHBEV_UNSUPPORTED = 2,  /* a combination this version does not implement (the tiled kernel on NCHW or
                                   on rows that are not whole 16-byte vectors, sizes beyond the index ranges
                                   stated below) */
-    FLASHBEV_MISALIGNED = 3,   /* `out` or `lidar2img` not 4-byte aligned, `features` not element aligned */
+    FLASHBEV_MISALIGNED = 3,   /* `out` or `lidar2img` not 4-byte aligned, `features` not element aligned (tensors that are
+                                  element- but not 16-byte aligned are served by the per-output kernel under AUTO and
+                                  refused with FLASHBEV_UNSUPPORTED under FLASHBEV_KERNEL_TILED) */
     FLASHBEV_CUDA_ERROR = 4,   /* the launch (or a copy of the host entry point) failed; the CUDA error
                                   has been consumed with cudaGetLastError */
     FLASHBEV_TOO_SMALL = 5,    /* a caller-provided staging buffer is smaller than required */
@@ -58,12 +62,14 @@ typedef enum flashbev_reduce {
 } flashbev_reduce;
 
 /* Kernel selection.  AUTO picks the tiled kernel whenever the channel row is a whole number of
- * 16-byte vectors and `features` is 16-byte aligned, the per-output kernel otherwise. */
+ * 16-byte vectors, `features` and `out` are 16-byte aligned and the shape is one the tiled kernel can
+ * be configured for; the per-output kernel (several times slower) otherwise --
+ * flashbev_last_kernel_name() tells which one ran. */
 typedef enum flashbev_kernel {
     FLASHBEV_KERNEL_AUTO = 0,
     FLASHBEV_KERNEL_PER_OUTPUT = 1, /* one thread per (cell, channel group), geometry recomputed per
                                        thread: the decomposition Algorithm 2 describes */
-    FLASHBEV_KERNEL_TILED = 2       /* geometry once per (cell, camera, height) per CTA, broadcast to
+    FLASHBEV_KERNEL_TILED = 2       /* geometry once per (cell, camera, height) per warp tile, handed to the
                                        channel lanes through shared memory */
 } flashbev_kernel;
 
@@ -82,7 +88,8 @@ typedef enum flashbev_kernel {
  *     taps is in bounds.
  * Projection, validity, floor and the fractional parts are evaluated in fp64; interpolation
  * weights and accumulation are fp32.  Non-finite matrix entries make the affected samples
- * invalid; they never cause a fault.
+ * invalid; they never cause a fault.  The forward result is reproducible bit for bit from run to
+ * run (no atomics, fixed summation order for a given launch configuration).
  *
  * Index ranges: N*feat_h*feat_w*C*sizeof(element) < 2^35 and B*X*Y < 2^31, N <= 64,
  * else FLASHBEV_UNSUPPORTED.
@@ -106,11 +113,21 @@ typedef struct flashbev_vt_params {
     int32_t out_dtype;         /* FLASHBEV_F32, or FLASHBEV_BF16: the fp32 result rounded to nearest even once */
     int32_t kernel;            /* flashbev_kernel */
     int32_t *valid_count_out;  /* optional [B][X][Y] int32: sum_z sum_n M_n per cell; NULL to skip */
-    int32_t tune[4];           /* 0 = library defaults.  tune[0]: channel vectors per lane (1,2,4);
-                                  tune[1]: lanes per cell; tune[2]: height bins per geometry walker;
-                                  tune[3]: bits 0-3 warps per CTA (1,2,4,8), bits 4-7 / 8-11 sub-blocks per warp in x / y,
-                                  bits 12-15 super-blocks per warp, bit 16 never / bit 17 always use 256-bit feature loads.
-                                  Invalid values fall back to the defaults */
+    int32_t tune[4];           /* launch-geometry hints of the tiled kernel, 0 = library defaults (they never change the
+                                  result beyond fp32 summation order).  tune[0]: channel vectors per lane (1,2,4);
+                                  tune[1]: lanes per cell; tune[2]: height bins (or texel rows) per geometry run, rounded
+                                  down to a power of two; tune[3]: bits 0-3 warps per CTA (1,2,4,8), bits 4-7 / 8-11
+                                  sub-blocks per warp in x / y, bits 12-15 super-blocks per warp, bit 16 never / bit 17
+                                  always use 256-bit feature loads, bits 18-19 super-block order (band height 4,1,2,8),
+                                  bits 20-27 record slots per warp in units of 16.  Values that do not fit fall back to
+                                  the defaults */
+    uint32_t *debug_error_word; /* optional DEVICE word, or NULL.  Only the bounds-checked build of the library
+                                  (-DFLASHBEV_DEBUG_BOUNDS) uses it: every shared-memory slot, record offset and
+                                  output index the tiled kernel computes is range-checked there; an index out of
+                                  range is counted into this word (atomically) and replaced by a safe one, never
+                                  dereferenced.  The caller zeroes the word before the call and reads it after
+                                  synchronising.  The normal build ignores it.  Callers built against an older
+                                  header (struct_size without this field) are accepted. */
 } flashbev_vt_params;
 
 /*
@@ -220,9 +237,9 @@ typedef struct flashbev_sca_params {
     const float *lidar2img;    /* device, [B][N][4][4] float32 */
     const float *offsets;      /* device, [B][X*Y][heads][L][P][2] float32, in texels of level l */
     const float *weights;      /* device, [B][X*Y][heads][L][P] float32 (normally a softmax over L*P) */
-    int32_t B, N, heads, head_dim; /* head_dim a multiple of 4 (float32) or 8 (bfloat16), <= 128; a head's
-                                      16-byte vectors must divide 32, at most 4 (float32) / 2 (bfloat16)
-                                      passes of 32 lanes over the heads: else FLASHBEV_UNSUPPORTED */
+    int32_t B, N, heads, head_dim; /* head_dim a multiple of 4 (float32) or 8 (bfloat16), <= 128; at most
+                                      4 (float32) / 2 (bfloat16) passes of 32 lanes over the heads (a head
+                                      takes head_dim * element size / 16 lanes): else FLASHBEV_UNSUPPORTED */
     int32_t L, P;
     int32_t img_h, img_w;
     double x_min, x_max;

@@ -43,6 +43,7 @@ class VtParams(ctypes.Structure):
         ("kernel", ctypes.c_int32),
         ("valid_count_out", ctypes.c_void_p),
         ("tune", ctypes.c_int32 * 4),
+        ("debug_error_word", ctypes.c_void_p),
     ]
 
 
@@ -110,6 +111,40 @@ class FlashBevError(RuntimeError):
 _lib = None
 
 
+def _declare(L: ctypes.CDLL) -> ctypes.CDLL:
+    """Argument and result types of every entry point of a loaded libflashbev."""
+    P = ctypes.POINTER(VtParams)
+    L.flashbev_sampling_vt.restype = ctypes.c_int
+    L.flashbev_sampling_vt.argtypes = [P, ctypes.c_void_p]
+    L.flashbev_sampling_vt_host.restype = ctypes.c_int
+    L.flashbev_sampling_vt_host.argtypes = [P, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    L.flashbev_sampling_vt_host_static.restype = ctypes.c_int
+    L.flashbev_sampling_vt_host_static.argtypes = [P, ctypes.c_void_p]
+    L.flashbev_sampling_vt_backward.restype = ctypes.c_int
+    L.flashbev_sampling_vt_backward.argtypes = [ctypes.POINTER(VtBackwardParams), ctypes.c_void_p]
+    L.flashbev_sampling_vt_multires.restype = ctypes.c_int
+    L.flashbev_sampling_vt_multires.argtypes = [ctypes.POINTER(VtMultiresParams), ctypes.c_void_p]
+    L.flashbev_sca.restype = ctypes.c_int
+    L.flashbev_sca.argtypes = [ctypes.POINTER(ScaParams), ctypes.c_void_p]
+    L.flashbev_workspace_bytes.restype = ctypes.c_size_t
+    L.flashbev_workspace_bytes.argtypes = [P]
+    L.flashbev_host_staging_bytes.restype = ctypes.c_size_t
+    L.flashbev_host_staging_bytes.argtypes = [P]
+    L.flashbev_last_launch_count.restype = ctypes.c_int
+    L.flashbev_last_kernel_name.restype = ctypes.c_char_p
+    L.flashbev_status_string.restype = ctypes.c_char_p
+    L.flashbev_status_string.argtypes = [ctypes.c_int]
+    L.flashbev_version.restype = ctypes.c_int
+    return L
+
+
+def load_library(path: str) -> ctypes.CDLL:
+    """Load another build of the library (e.g. the bounds-checked one) next to the default one."""
+    if not os.path.exists(path):
+        raise FileNotFoundError(f"{path} is missing: build it with paper_2607_10071_b200.build (there is no CPU fallback)")
+    return _declare(ctypes.CDLL(path))
+
+
 def lib() -> ctypes.CDLL:
     """Load libflashbev.so (built in-tree by ``paper_2607_10071_b200.build``)."""
     global _lib
@@ -118,30 +153,7 @@ def lib() -> ctypes.CDLL:
             raise FileNotFoundError(
                 f"{LIB_PATH} is missing: build it with `python -m paper_2607_10071_b200.build` "
                 "(there is no CPU fallback)")
-        L = ctypes.CDLL(LIB_PATH)
-        P = ctypes.POINTER(VtParams)
-        L.flashbev_sampling_vt.restype = ctypes.c_int
-        L.flashbev_sampling_vt.argtypes = [P, ctypes.c_void_p]
-        L.flashbev_sampling_vt_host.restype = ctypes.c_int
-        L.flashbev_sampling_vt_host.argtypes = [P, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
-        L.flashbev_sampling_vt_host_static.restype = ctypes.c_int
-        L.flashbev_sampling_vt_host_static.argtypes = [P, ctypes.c_void_p]
-        L.flashbev_sampling_vt_backward.restype = ctypes.c_int
-        L.flashbev_sampling_vt_backward.argtypes = [ctypes.POINTER(VtBackwardParams), ctypes.c_void_p]
-        L.flashbev_sampling_vt_multires.restype = ctypes.c_int
-        L.flashbev_sampling_vt_multires.argtypes = [ctypes.POINTER(VtMultiresParams), ctypes.c_void_p]
-        L.flashbev_sca.restype = ctypes.c_int
-        L.flashbev_sca.argtypes = [ctypes.POINTER(ScaParams), ctypes.c_void_p]
-        L.flashbev_workspace_bytes.restype = ctypes.c_size_t
-        L.flashbev_workspace_bytes.argtypes = [P]
-        L.flashbev_host_staging_bytes.restype = ctypes.c_size_t
-        L.flashbev_host_staging_bytes.argtypes = [P]
-        L.flashbev_last_launch_count.restype = ctypes.c_int
-        L.flashbev_last_kernel_name.restype = ctypes.c_char_p
-        L.flashbev_status_string.restype = ctypes.c_char_p
-        L.flashbev_status_string.argtypes = [ctypes.c_int]
-        L.flashbev_version.restype = ctypes.c_int
-        _lib = L
+        _lib = _declare(ctypes.CDLL(LIB_PATH))
     return _lib
 
 
@@ -155,7 +167,7 @@ def version() -> int:
 
 def make_params(features_ptr, feat_dtype, lidar2img_ptr, B, N, C, feat_hw, img_hw, bev_range, grid,
                 reduce, out_ptr, valid_count_ptr=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0),
-                layout=NHWC, out_dtype=F32) -> VtParams:
+                layout=NHWC, out_dtype=F32, debug_error_word=None) -> VtParams:
     p = VtParams()
     p.struct_size = ctypes.sizeof(VtParams)
     p.features, p.feat_dtype, p.layout = features_ptr, feat_dtype, layout
@@ -168,14 +180,16 @@ def make_params(features_ptr, feat_dtype, lidar2img_ptr, B, N, C, feat_hw, img_h
     p.reduce = reduce
     p.out, p.out_dtype, p.kernel = out_ptr, out_dtype, kernel
     p.valid_count_out = valid_count_ptr
+    p.debug_error_word = debug_error_word
     for i, t in enumerate(tune):
         p.tune[i] = int(t)
     return p
 
 
-def flashbev_sampling_vt(params: VtParams, stream: int | None = None, check: bool = True) -> int:
-    """Enqueue the fused operator on ``stream`` (a raw cudaStream_t value; None/0 = default stream)."""
-    st = lib().flashbev_sampling_vt(ctypes.byref(params), ctypes.c_void_p(stream or 0))
+def flashbev_sampling_vt(params: VtParams, stream: int | None = None, check: bool = True, library=None) -> int:
+    """Enqueue the fused operator on ``stream`` (a raw cudaStream_t value; None/0 = default stream).
+    ``library``: another build loaded with ``load_library`` instead of the default one."""
+    st = (library or lib()).flashbev_sampling_vt(ctypes.byref(params), ctypes.c_void_p(stream or 0))
     if check and st != OK:
         raise FlashBevError(st, "flashbev_sampling_vt")
     return st
@@ -236,9 +250,10 @@ def make_backward_params(grad_out_ptr, lidar2img_ptr, B, N, C, feat_hw, img_hw, 
     return p
 
 
-def flashbev_sampling_vt_backward(params: VtBackwardParams, stream: int | None = None, check: bool = True) -> int:
+def flashbev_sampling_vt_backward(params: VtBackwardParams, stream: int | None = None, check: bool = True,
+                                  library=None) -> int:
     """Enqueue the gradient w.r.t. the features (memset + one scatter kernel) on ``stream``."""
-    st = lib().flashbev_sampling_vt_backward(ctypes.byref(params), ctypes.c_void_p(stream or 0))
+    st = (library or lib()).flashbev_sampling_vt_backward(ctypes.byref(params), ctypes.c_void_p(stream or 0))
     if check and st != OK:
         raise FlashBevError(st, "flashbev_sampling_vt_backward")
     return st

@@ -22,9 +22,12 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
+#include <string.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 
 namespace {
@@ -63,7 +66,6 @@ struct KParams {
     int rstep;                  // distance (16-byte vectors) from a record's first tap to its second: vecs, or 0 on 1-texel-wide maps
     int nvec_cam;               // N * Hf * Wf * vecs: vectors of one batch element's feature maps (bounds-checked build)
     int wide;                   // host side: use the instance with adjacent channel vectors and 256-bit loads
-    int dbg;
     unsigned *err;              // bounds-checked build: device word that counts out-of-range indices (may be null)
 };
 
@@ -208,7 +210,7 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
         }
         count += den;
         if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) {
-            const float g = 1.f / (float)(den > 1 ? den : 1);  // g_z = num_z / max(1, den_z)
+            const float g = 1.f / (float)(den > 1 ? den : 1);  // mean over the cameras that see this height
 #pragma unroll
             for (int i = 0; i < VEC; ++i) acc[i] = fmaf(num[i], g, acc[i]);
         } else {
@@ -570,10 +572,26 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
 thread_local int t_last_launches = 0;
 thread_local const char *t_last_kernel = "none";
 
+// The optional device word of the bounds-checked build (absent in structs of callers built against an older header).
+unsigned *debug_word(const flashbev_vt_params *p)
+{
+    return p->struct_size >= sizeof(flashbev_vt_params) ? p->debug_error_word : nullptr;
+}
+
+// A full-size copy of a caller's struct, which may be shorter (older header): missing fields are zero.
+flashbev_vt_params copy_params(const flashbev_vt_params *p)
+{
+    flashbev_vt_params c;
+    memset(&c, 0, sizeof(c));
+    memcpy(&c, p, std::min(p->struct_size, sizeof(c)));
+    c.struct_size = sizeof(c);
+    return c;
+}
+
 bool params_ok(const flashbev_vt_params *p, flashbev_status &st)
 {
     st = FLASHBEV_INVALID_ARG;
-    if (!p || p->struct_size < sizeof(flashbev_vt_params)) return false;
+    if (!p || p->struct_size < offsetof(flashbev_vt_params, debug_error_word)) return false;  // (older headers end there)
     if (!p->features || !p->lidar2img || !p->out) return false;
     if (p->B <= 0 || p->N <= 0 || p->C <= 0 || p->feat_h <= 0 || p->feat_w <= 0 || p->img_h <= 0 || p->img_w <= 0)
         return false;
@@ -604,6 +622,7 @@ flashbev_status check_alignment(const flashbev_vt_params *p)
     const size_t oelem = p->out_dtype == FLASHBEV_F32 ? 4 : 2;
     if (((uintptr_t)p->features % elem) || ((uintptr_t)p->out % oelem) || ((uintptr_t)p->lidar2img % 4)) return FLASHBEV_MISALIGNED;
     if (p->valid_count_out && ((uintptr_t)p->valid_count_out % 4)) return FLASHBEV_MISALIGNED;
+    if (debug_word(p) && ((uintptr_t)debug_word(p) % 4)) return FLASHBEV_MISALIGNED;
     return FLASHBEV_OK;
 }
 
@@ -618,6 +637,7 @@ KParams base_params(const flashbev_vt_params *p, bool accumulate = false)
     k.B = p->B, k.N = p->N, k.C = p->C, k.Hf = p->feat_h, k.Wf = p->feat_w;
     k.X = p->X, k.Y = p->Y, k.Z = p->Z, k.reduce = p->reduce;
     k.out_bf16 = p->out_dtype == FLASHBEV_BF16;
+    k.err = debug_word(p);
     k.sx = (double)p->feat_w / (double)p->img_w;
     k.sy = (double)p->feat_h / (double)p->img_h;
     k.x_min = p->x_min, k.dx = (p->x_max - p->x_min) / (double)p->X;
@@ -665,21 +685,21 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
 // Number of SMs of the current device (cached per device; 148 on a B200).
 int sm_count()
 {
-    static int cached[64];
+    static std::atomic<int> cached[64];  // 0: not asked yet (concurrent callers may both ask: same answer)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
         cudaGetLastError();
         return 148;
     }
-    if (!cached[dev]) {
-        int n = 0;
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (!n) {
         if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
             cudaGetLastError();
             n = 148;
         }
-        cached[dev] = n;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
-    return cached[dev];
+    return n;
 }
 
 bool tiled_applicable(const flashbev_vt_params *p)
@@ -731,7 +751,6 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     k.rstep = p->feat_w > 1 ? k.vecs : 0;
     k.nvec_cam = p->N * p->feat_h * p->feat_w * k.vecs;  // < 2^31: tiled_applicable
     k.inv_n = 1.0f / (float)p->N;
-    k.dbg = (p->tune[3] >> 28) & 15;
 
     // channel mapping: V vectors per lane, g lanes per cell
     V = p->tune[0];
@@ -857,6 +876,8 @@ flashbev_status run_device(const flashbev_vt_params *p, cudaStream_t stream, boo
     const bool tiled = p->kernel == FLASHBEV_KERNEL_TILED || (p->kernel == FLASHBEV_KERNEL_AUTO && tiled_applicable(p));
     if (tiled && !tiled_applicable(p)) return FLASHBEV_UNSUPPORTED;
     st = tiled ? launch_tiled(p, stream, accumulate) : launch_per_output(p, stream, accumulate);
+    // AUTO: shapes the tiled kernel cannot be configured for (nothing was launched) go to the generic kernel
+    if (tiled && st == FLASHBEV_UNSUPPORTED && p->kernel == FLASHBEV_KERNEL_AUTO) st = launch_per_output(p, stream, accumulate);
     if (st != FLASHBEV_OK) return st;
     if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
     t_last_launches = 1;
@@ -867,17 +888,20 @@ struct StagingLayout {
     size_t feat_off, mat_off, out_off, cnt_off, total;
 };
 
-StagingLayout staging_layout(const flashbev_vt_params *p)
+// False if the staging area of this problem would not fit 2^62 bytes (the byte counts below would wrap).
+bool staging_layout(const flashbev_vt_params *p, StagingLayout &s)
 {
-    auto up = [](size_t v) { return (v + 255) / 256 * 256; };
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
-    StagingLayout s;
+    const double feat = (double)p->B * p->N * p->feat_h * p->feat_w * p->C * (double)elem;
+    const double out = (double)p->B * p->X * p->Y * p->C * 4.0;
+    if (!(feat + out + (double)p->B * p->N * 64.0 + (double)p->B * p->X * p->Y * 4.0 < 4.0e18)) return false;
+    auto up = [](size_t v) { return (v + 255) / 256 * 256; };
     s.feat_off = 0;
     s.mat_off = up((size_t)p->B * p->N * p->feat_h * p->feat_w * p->C * elem);
     s.out_off = s.mat_off + up((size_t)p->B * p->N * 64);
     s.cnt_off = s.out_off + up((size_t)p->B * p->X * p->Y * p->C * (p->out_dtype == FLASHBEV_F32 ? 4 : 2));
     s.total = s.cnt_off + (p->valid_count_out ? up((size_t)p->B * p->X * p->Y * 4) : 0);
-    return s;
+    return true;
 }
 
 }  // namespace
@@ -902,7 +926,8 @@ size_t flashbev_host_staging_bytes(const flashbev_vt_params *p)
 {
     flashbev_status st;
     if (!params_ok(p, st)) return 0;
-    return staging_layout(p).total;
+    StagingLayout L;
+    return staging_layout(p, L) ? L.total : 0;
 }
 
 flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_staging, size_t staging_bytes,
@@ -912,11 +937,12 @@ flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_s
     if (!params_ok(p, st)) return st;
     if (!d_staging) return FLASHBEV_INVALID_ARG;
     if ((uintptr_t)d_staging % 256) return FLASHBEV_MISALIGNED;
-    const StagingLayout L = staging_layout(p);
+    StagingLayout L;
+    if (!staging_layout(p, L)) return FLASHBEV_UNSUPPORTED;
     if (staging_bytes < L.total) return FLASHBEV_TOO_SMALL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     unsigned char *base = static_cast<unsigned char *>(d_staging);
-    flashbev_vt_params d = *p;
+    flashbev_vt_params d = copy_params(p);
     d.features = base + L.feat_off;
     d.lidar2img = reinterpret_cast<const float *>(base + L.mat_off);
     d.out = base + L.out_off;
@@ -995,12 +1021,11 @@ flashbev_status flashbev_sampling_vt_multires(const flashbev_vt_multires_params 
     if (!q || q->struct_size < sizeof(flashbev_vt_multires_params) || !q->base || !q->features || !q->feat_hw)
         return FLASHBEV_INVALID_ARG;
     if (q->levels < 1 || q->levels > FLASHBEV_MAX_LEVELS) return FLASHBEV_INVALID_ARG;
-    if (q->base->struct_size < sizeof(flashbev_vt_params)) return FLASHBEV_INVALID_ARG;
+    if (q->base->struct_size < offsetof(flashbev_vt_params, debug_error_word)) return FLASHBEV_INVALID_ARG;
     flashbev_vt_params lv[FLASHBEV_MAX_LEVELS];
     flashbev_status st;
     for (int l = 0; l < q->levels; ++l) {  // every level is checked before anything is enqueued
-        lv[l] = *q->base;
-        lv[l].struct_size = sizeof(flashbev_vt_params);
+        lv[l] = copy_params(q->base);
         lv[l].features = q->features[l];
         lv[l].feat_h = q->feat_hw[2 * l], lv[l].feat_w = q->feat_hw[2 * l + 1];
         if (l > 0) lv[l].valid_count_out = nullptr;
@@ -1131,7 +1156,8 @@ flashbev_status flashbev_sampling_vt_host_static(const flashbev_vt_params *p, vo
 {
     flashbev_status st;
     if (!params_ok(p, st)) return st;
-    if (staging_layout(p).total > (size_t)FLASHBEV_STATIC_STAGING_BYTES) return FLASHBEV_EXCEEDS_STATIC_STAGING;
+    StagingLayout L;
+    if (!staging_layout(p, L) || L.total > (size_t)FLASHBEV_STATIC_STAGING_BYTES) return FLASHBEV_EXCEEDS_STATIC_STAGING;
     void *staging = static_staging_address();  // first call on this device: symbol look-up
     if (!staging) return FLASHBEV_CUDA_ERROR;
     // From here on this is the caller-staged path with the built-in area as the staging buffer.

@@ -413,6 +413,9 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
 
     if (affine_by_rows(D)) {
         len = min(len, cap);  // (never cuts: the run's slots were counted from the same numbers)
+#ifdef FLASHBEV_DEBUG_BOUNDS
+        (void)FB_IDX((out_off - sm.roff) + len - 1, p.slots, p.err);
+#endif
         const int ra = max((int)floor(A), 0) + u0;
         const double inv = (double)__frcp_rn((float)S);
         auto first_bin_at = [&](double rr) {  // smallest k' in [0, nb] with A + k' S >= rr
@@ -433,6 +436,9 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
             const int i = (int)fl - ra;  // row of the upper tap, relative
             float ty = (float)(fy - fl), tu = 1.f - ty;
             if (eq1) {
+#ifdef FLASHBEV_DEBUG_BOUNDS
+                dk = sm.den + FB_IDX(dk - sm.den, p.den_bytes, p.err);
+#endif
                 const float sc = 1.f / (float)max(1, (int)*dk);
                 ty *= sc, tu *= sc;
             }
@@ -448,6 +454,9 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
     } else {
         // rows of successive bins never coincide: two records per bin (a row outside the map: weight 0, clamped)
         len = min(len, cap / 2);
+#ifdef FLASHBEV_DEBUG_BOUNDS
+        (void)FB_IDX((out_off - sm.roff) + 2 * len - 1, p.slots, p.err);
+#endif
         double kd = (double)u0;
         const unsigned char *dk = den + u0 * dstep;
         for (int i = 0; i < len; ++i, kd += 1.0, dk += dstep) {
@@ -455,6 +464,9 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
             const int r = (int)fl;
             float ty = (float)(fy - fl), tu = 1.f - ty;
             if (eq1) {
+#ifdef FLASHBEV_DEBUG_BOUNDS
+                dk = sm.den + FB_IDX(dk - sm.den, p.den_bytes, p.err);
+#endif
                 const float sc = 1.f / (float)max(1, (int)*dk);
                 ty *= sc, tu *= sc;
             }
@@ -773,13 +785,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
             in_mask = __ballot_sync(FULL, in);
         }
         __syncwarp();
-        if (p.dbg & 8) {
-            sm.cfirst[lane] = 0;
-            if (lane == 0) sm.cfirst[32] = 0;
-            __syncwarp();
-        } else {
-            survey_candidates(p, cx, in_mask);
-        }
+        survey_candidates(p, cx, in_mask);
 
         // ---- segments: as many sub-blocks as have at most `colcap` surviving columns together (normally all of them)
         for (int s0 = 0; s0 < p.sbn;) {
@@ -787,7 +793,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
             int s1 = s0 + 1;
             while (s1 < p.sbn && sm.cfirst[min((s1 + 1) * p.cpw, p.ct)] - jb <= p.colcap) ++s1;
             const int ncols = sm.cfirst[min(s1 * p.cpw, p.ct)] - jb;  // <= colcap: a sub-block has at most cpw * N candidates
-            const int nw = (p.dbg & 4) ? 0 : build_columns(p, cx, jb, ncols, s0 * p.cpw, min(s1 * p.cpw, p.ct));
+            const int nw = build_columns(p, cx, jb, ncols, s0 * p.cpw, min(s1 * p.cpw, p.ct));
 
             // ---- rounds: the runs of as many whole sub-blocks as fit the record slots are walked together (one lane
             // per run), then the sub-blocks are gathered one by one
@@ -799,9 +805,8 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                 // (lanes without a cell inside the grid never use it)
                 const size_t ocell = lane_on ? (size_t)FB_IDX(((size_t)b * p.X + (ix0 + (tab & 0xff))) * p.Y + (iy0 + (tab >> 8)),
                                                               (size_t)p.B * p.X * p.Y, p.err) : 0;
-                int sw_lo = sm.colw[sm.cfirst[s * p.cpw] - jb], sw_hi = sm.colw[sm.cfirst[min((s + 1) * p.cpw, p.ct)] - jb];
-                int cw_lo = sm.colw[sm.cfirst[cell] - jb], cw_hi = sm.colw[sm.cfirst[cell + 1] - jb];  // this lane's cell
-                if (p.dbg & 4) sw_lo = sw_hi = cw_lo = cw_hi = 0;
+                const int sw_lo = sm.colw[sm.cfirst[s * p.cpw] - jb], sw_hi = sm.colw[sm.cfirst[min((s + 1) * p.cpw, p.ct)] - jb];
+                const int cw_lo = sm.colw[sm.cfirst[cell] - jb], cw_hi = sm.colw[sm.cfirst[cell + 1] - jb];  // this lane's cell
                 const int sub_records = sm.woff[sw_hi] - sm.woff[sw_lo];
                 const bool oversized = sub_records > p.slots;
                 if (!oversized && sw_hi > wb) {
@@ -813,7 +818,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                         wb = hi2;
                     }
                     const int base = sm.woff[wa];
-                    for (int w = wa + lane; w < wb && !(p.dbg & 2); w += 32) walk_one(p, sm, mats, w, sm.woff[w] - base);
+                    for (int w = wa + lane; w < wb; w += 32) walk_one(p, sm, mats, w, sm.woff[w] - base);
                     __syncwarp();
                 }
 
@@ -841,7 +846,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
 
                 if (!oversized) {
                     const int c0 = sm.woff[cw_lo] - sm.woff[wa];
-                    const int nrec = (lane_on && !(p.dbg & 1)) ? sm.woff[cw_hi] - sm.woff[cw_lo] : 0;
+                    const int nrec = lane_on ? sm.woff[cw_hi] - sm.woff[cw_lo] : 0;
                     if (BWD) {
                         if (nrec > 0) scatter_list<V>(go, on, sm.roff + c0, sm.rw + c0, nrec, p.rstep, gfv);
                     } else {
@@ -863,12 +868,12 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                             if (bal != FULL) break;
                         }
                         if (upto <= pos) upto = pos + 1;  // (cannot happen: one run always fits; never loop without progress)
-                        for (int w = pos + lane; w < upto && !(p.dbg & 2); w += 32) walk_one(p, sm, mats, w, sm.woff[w] - base);
+                        for (int w = pos + lane; w < upto; w += 32) walk_one(p, sm, mats, w, sm.woff[w] - base);
                         __syncwarp();
                         // this lane's cell: its runs inside [pos, upto)
                         const int lw = min(max(cw_lo, pos), upto), hw = min(max(cw_hi, pos), upto);
                         const int c0 = sm.woff[lw] - base;
-                        const int nrec = (lane_on && !(p.dbg & 1)) ? sm.woff[hw] - sm.woff[lw] : 0;
+                        const int nrec = lane_on ? sm.woff[hw] - sm.woff[lw] : 0;
                         if (BWD) {
                             if (nrec > 0) scatter_list<V>(go, on, sm.roff + c0, sm.rw + c0, nrec, p.rstep, gfv);
                         } else {

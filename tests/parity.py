@@ -77,7 +77,10 @@ def compare(w, ref, out, count) -> ParityReport:
                         int(ref.count.sum()))
 
 
-def assert_parity(w, ref, out, count, label="", check_fraction=True):
+def assert_parity(w, ref, out, count, label="", check_fraction=True, large_outputs=False):
+    """large_outputs: stress cases with hundreds of samples per cell reach |out| far above the 1-10 the absolute
+    fp32 bound was stated for (fp32 accumulation error grows with |out|): there the absolute bound is taken
+    relative to the output scale, 1e-4 * max(1, max|ref| / 10); the relative-L2 bound is unchanged."""
     rep = compare(w, ref, out, count)
     msg = f"{label} {w.name}: {rep}"
     assert np.all(np.isfinite(out)), f"{msg}: output has non-finite or unwritten elements"
@@ -85,7 +88,8 @@ def assert_parity(w, ref, out, count, label="", check_fraction=True):
     if check_fraction:
         assert rep.flagged_fraction < MAX_FLAGGED_FRACTION, msg
     if w.dtype == "f32":
-        assert rep.max_abs <= F32_MAX_ABS, msg
+        scale = max(1.0, float(np.abs(ref.out).max()) / 10.0) if large_outputs else 1.0
+        assert rep.max_abs <= F32_MAX_ABS * scale, f"{msg} (bound {F32_MAX_ABS * scale:.2e})"
         assert rep.rel_l2 <= F32_REL_L2, msg
     else:
         assert rep.worst_bf16_ratio <= 1.0, msg

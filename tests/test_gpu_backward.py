@@ -51,6 +51,14 @@ def test_backward_benchmark_shapes(oracle, name, reduce):
     print("\n" + check(oracle, w, inp.lidar2img, reduce))
 
 
+def test_backward_long_range_shape_fp32(oracle):
+    """The largest benchmark grid with 128 fp32 channels: many sub-blocks per warp, 32-vector texels, record
+    offsets beyond 2^20 (the forward benchmark uses bf16 there; the backward is fp32 only)."""
+    w = wl.get("long_range", dtype="f32")
+    inp = wl.make_inputs(w)
+    print("\n" + check(oracle, w, inp.lidar2img, SUM))
+
+
 @pytest.mark.parametrize("reduce", [SUM, MEAN, EQ1])
 @pytest.mark.parametrize("C", [4, 36, 80, 128, 260])
 def test_backward_general_pose_channel_counts(oracle, reduce, C):

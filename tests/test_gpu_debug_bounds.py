@@ -1,0 +1,94 @@
+"""The bounds-checked build of the CUDA library (-DFLASHBEV_DEBUG_BOUNDS) on a GPU.
+
+No memory checker may run on the shared machines, so the library can be built with its own guard: every
+shared-memory slot, record offset and output index the tiled kernel computes goes through a range check that
+counts a violation into the caller's ``debug_error_word`` and redirects the access to a safe slot.  These tests
+run the benchmark configurations, the many-rounds stress case, odd shapes and the backward pass in that build,
+require the word to stay 0 and the results to match the oracle as in the normal build.
+"""
+import numpy as np
+import pytest
+
+from paper_2607_10071_b200 import binding as fb
+from paper_2607_10071_b200 import build as fbuild
+from paper_2607_10071_b200 import workloads as wl
+from tests import parity
+from tests.test_gpu_parity import small
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def checked():
+    return fb.load_library(fbuild.build(debug_bounds=True))
+
+
+def run_checked(checked, inp, reduce, tune=(0, 0, 0, 0)):
+    import torch
+    w = inp.workload
+    dev = torch.device("cuda:0")
+    if w.dtype == "bf16":
+        feats = torch.from_numpy(inp.features_bf16.view(np.int16)).to(dev).view(torch.bfloat16)
+    else:
+        feats = torch.from_numpy(inp.features).to(dev)
+    mats = torch.from_numpy(inp.lidar2img).to(dev)
+    X, Y, Z = w.grid
+    out = torch.full((w.B, X, Y, w.C), float("nan"), dtype=torch.float32, device=dev)
+    cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=dev)
+    word = torch.zeros(1, dtype=torch.int32, device=dev)
+    p = fb.make_params(feats.data_ptr(), fb.BF16 if w.dtype == "bf16" else fb.F32, mats.data_ptr(), w.B, w.N, w.C,
+                       w.feat_hw, w.img_hw, w.bev_range, w.grid, reduce, out.data_ptr(), cnt.data_ptr(), fb.KERNEL_TILED,
+                       tune, debug_error_word=word.data_ptr())
+    fb.flashbev_sampling_vt(p, torch.cuda.current_stream().cuda_stream, library=checked)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), cnt.cpu().numpy(), int(word.item())
+
+
+@pytest.mark.parametrize("name", wl.CONFIG_ORDER)
+def test_benchmark_configurations_make_no_out_of_range_index(oracle, checked, name):
+    inp = wl.make_inputs(wl.get(name))
+    w = inp.workload
+    for reduce in {w.reduce, 2}:
+        out, cnt, violations = run_checked(checked, inp, reduce)
+        assert violations == 0, f"{name} reduce={reduce}: {violations} out-of-range indices"
+        ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, reduce)
+        parity.assert_parity(w, ref, out, cnt, f"[bounds-checked build, reduce={reduce}]")
+
+
+def test_many_rounds_and_odd_shapes_make_no_out_of_range_index(oracle, checked):
+    # all cameras overlap: far more records per cell than the slots hold
+    w = wl.Workload("overlap", 77, 1, 8, 32, "f32", (24, 40), (192, 320), (12, 10, 96),
+                    (8.0, 20.0, -5.0, 5.0, -2.0, 4.0), 0, general_pose=False, yaw_jitter_deg=0.0)
+    inp = wl.make_inputs(w)
+    inp.lidar2img[:] = inp.lidar2img[:, :1]
+    inp.lidar2img[0, :, 0, 3] += np.arange(8, dtype=np.float32) * 3.0
+    cases = [(inp, 2, (0, 0, 0, 0)), (inp, 0, (0, 0, 4, 0x04000000)), (inp, 1, (0, 0, 64, 0))]
+    for seed, kw in ((1, dict(grid=(1, 1, 1))), (2, dict(grid=(33, 31, 7), C=80)), (3, dict(feat=(1, 1))),
+                     (4, dict(feat=(12, 1))), (5, dict(N=33, C=16, grid=(10, 9, 6))), (6, dict(grid=(9, 11, 300), B=1)),
+                     (7, dict(C=128, dtype="bf16", general=False, grid=(40, 40, 12), rng_xy=30.0)),
+                     (8, dict(C=260)), (9, dict(C=264, dtype="bf16"))):
+        cases.append((small(700 + seed, **kw), 2, (0, 0, 0, 0)))
+    for case, reduce, tune in cases:
+        out, cnt, violations = run_checked(checked, case, reduce, tune)
+        assert violations == 0, f"{case.workload.name} {case.workload.grid} reduce={reduce} tune={tune}: {violations}"
+        assert np.all(np.isfinite(out))
+        assert cnt.min() >= 0
+
+
+def test_backward_makes_no_out_of_range_index(checked):
+    """The backward entry point has no error-word field: run it in the checked build for its clamping only and
+    compare with the normal build (the scatter order differs from run to run, hence a tolerance)."""
+    import torch
+    w = wl.get("tiny")
+    inp = wl.make_inputs(w)
+    dev = torch.device("cuda:0")
+    X, Y, Z = w.grid
+    go = torch.randn((w.B, X, Y, w.C), generator=torch.Generator().manual_seed(3)).to(dev)
+    mats = torch.from_numpy(inp.lidar2img).to(dev)
+    ref = fb.sampling_vt_backward(go, mats, w.feat_hw, w.img_hw, w.bev_range, w.grid, 2)
+    gf = torch.empty_like(ref)
+    p = fb.make_backward_params(go.data_ptr(), mats.data_ptr(), w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid, 2,
+                                gf.data_ptr())
+    fb.flashbev_sampling_vt_backward(p, torch.cuda.current_stream().cuda_stream, library=checked)
+    torch.cuda.synchronize()
+    assert torch.allclose(gf, ref, rtol=1e-5, atol=1e-5)

@@ -34,9 +34,6 @@ def test_random_small_problems_match_the_oracle(oracle, case):
                     (-case["rng_xy"], case["rng_xy"], -case["rng_xy"], case["rng_xy"], -3.0, 2.5), case["reduce"],
                     general_pose=case["general"], yaw_jitter_deg=5.0)
     inp = wl.make_inputs(w)
-    inp.features *= np.float32(0.25)          # |out| of order one even with ~200 samples per cell
-    if inp.features_bf16 is not None:
-        inp.features, inp.features_bf16 = wl.round_to_bf16(inp.features)
     ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, case["reduce"])
     out, cnt, kname = parity.run_gpu(inp, case["reduce"], case["kernel"], (0, 0, case["walk"], 0))
-    parity.assert_parity(w, ref, out, cnt, f"[{kname} {case}]", check_fraction=False)
+    parity.assert_parity(w, ref, out, cnt, f"[{kname} {case}]", check_fraction=False, large_outputs=True)  # up to ~200 samples per cell

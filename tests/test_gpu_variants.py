@@ -74,8 +74,7 @@ def test_bf16_output_is_the_fp32_result_rounded_once(oracle, kernel, name, reduc
     assert np.all(err[keep] <= bound[keep]), float((err / bound)[keep].max())
     # and it is exactly the rounding of the fp32 output of the same kernel
     out32 = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, kernel=kernel)
-    if kernel == fb.KERNEL_PER_OUTPUT:
-        assert torch.equal(out32.to(torch.bfloat16), out)
+    assert torch.equal(out32.to(torch.bfloat16), out)   # (both kernels: same sums, one rounding at the store)
 
 
 def test_bf16_output_with_nchw(oracle):

@@ -238,6 +238,47 @@ def test_tiny_workload_counts_match_tensorized_geometry(oracle):
     assert np.allclose(r.out, ref, rtol=0, atol=1e-11)
 
 
+def zero_jitter_totals():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "zero_jitter_valid_totals.txt")) if l.strip() and not l.startswith("#")]
+    return {r[0]: (int(r[1]), int(r[2])) for r in rows}
+
+
+@pytest.mark.parametrize("name", ["tiny", "representative", "half_taller"])
+def test_valid_sample_totals_of_the_benchmark_rigs_without_jitter(oracle, name):
+    """Geometry + validity at full grid size: the totals of an independent enumeration (a handful of samples
+    within 1e-3 px of a border may fall either way; the oracle flags those)."""
+    cand, valid = zero_jitter_totals()[name]
+    w = wl.get(name, yaw_jitter_deg=0.0, C=4 if wl.get(name).dtype == "f32" else 8)
+    inp = wl.make_inputs(w)
+    r = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, SUM)
+    assert w.candidates == cand
+    assert abs(int(r.count.sum()) - valid) <= int(r.flagged.sum())
+    assert r.flagged.sum() <= 1e-4 * cand
+
+
+def test_height_bins_seen_by_hand(oracle):
+    """nzbins counts the height bins seen by at least one camera; count adds the cameras up.
+    One cell, three bins z = 0.5, 1.5, 2.5, image 8 x 12, map 4 x 6, orthographic cameras (depth 1):
+      A: u = 20 z - 15 = -5, 15, 35 -> always outside 0 < u < 12: sees no bin;
+      B: u = 6, v = 2 z + 1 = 2, 4, 6 -> sees all three;
+      C: u = 6, v = 4 z - 1 = 1, 5, 9 -> sees bins 0 and 1 (9 > 8).
+    So count = 5 and nzbins = 3."""
+    A = ortho(0.0, -15.0, 0.0, 1.0, gu=20.0, gv=2.0)
+    Bm = ortho(0.0, 6.0, 0.0, 1.0, gv=2.0)
+    Cm = ortho(0.0, 6.0, 0.0, -1.0, gv=4.0)
+    M = np.stack([A, Bm, Cm])[None]
+    F = np.ones((1, 3, 4, 6, 1), np.float32)
+    r = oracle.sampling_vt(F, M, (8, 12), (0, 1, 0, 1, 0, 3), (1, 1, 3), SUM)
+    assert r.count[0, 0, 0] == 5 and r.nzbins[0, 0, 0] == 3
+    # constant map, all samples interior: SUM = count, Eq. 1 = bins seen, MEAN = 1
+    assert r.out[0, 0, 0, 0] == pytest.approx(5.0, abs=1e-12)
+    e = oracle.sampling_vt(F, M, (8, 12), (0, 1, 0, 1, 0, 3), (1, 1, 3), EQ1)
+    assert e.out[0, 0, 0, 0] == pytest.approx(3.0, abs=1e-12)
+    # drop camera B: bins 0 and 1 are seen once, bin 2 never
+    r2 = oracle.sampling_vt(F[:, [0, 2]], M[:, [0, 2]], (8, 12), (0, 1, 0, 1, 0, 3), (1, 1, 3), SUM)
+    assert r2.count[0, 0, 0] == 2 and r2.nzbins[0, 0, 0] == 2
+
+
 # ---------------------------------------------------------------- invariants of Eq. 1
 
 @pytest.fixture(scope="module")

@@ -35,9 +35,15 @@ if ROOT not in sys.path:
 from paper_2607_10071_b200 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (bytes; None where no capture of that workload exists)
-NCU_DRAM_TRAFFIC = {"representative": 4.76e6, "long_range": 42.40e6}
+MIN_LAUNCHES_PER_STEP = 64
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (bytes), from ncu captures of single
+# launches taken from the middle of a step of rotating frames -- the regime that is timed -- summarised under
+# profiles/vt_tiled_kernel_<workload>.md.  The output of a launch is still partly in the 126 MB L2 when its kernel
+# ends, so these figures can lie below the algorithmic bytes: see `traffic_note` in the JSON line.
+NCU_DRAM_TRAFFIC = {"tiny": 0.336e6, "representative": 4.78e6, "half_taller": 8.26e6, "long_range": 40.71e6, "high_res": 24.78e6}
+TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum of one launch captured in the middle of a rotating-frame "
+                "step (ncu, one pass); part of a launch's output is written back from L2 after its kernel ends, so the "
+                "figure can be below the algorithmic bytes")
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "fused_sampling_vt_throughput"
 UNIT = "sample-channels/s"
@@ -109,7 +115,9 @@ def whole_job_value(total_ms_local: float, units_per_rank: float, world: int, re
 
 
 def frames_for(w: wl.Workload, min_bytes: int) -> int:
-    return max(4, -(-min_bytes // w.unique_bytes))
+    """Frames per step: their inputs and outputs together exceed `min_bytes` (L2-cold launches without a flush), and
+    there are enough launches for the timed region of a step to be milliseconds long."""
+    return max(MIN_LAUNCHES_PER_STEP, -(-min_bytes // w.unique_bytes))
 
 
 def oracle_throughput(w: wl.Workload, seconds_budget: float, max_frames: int):
@@ -173,13 +181,12 @@ class DeviceFrames:
         X, Y, Z = w.grid
         self.feats, self.mats, self.outs, self.params = [], [], [], []
         base = wl.make_inputs(w, stream=1000 * rank)
-        g = torch.Generator(device="cpu").manual_seed(2607_10071 + rank)
+        g = torch.Generator(device=device).manual_seed(2607_10071 + rank)
         for i in range(frames):
             if i == 0:
-                f32 = torch.from_numpy(base.features)
-            else:  # same shape and distribution, different values (standard normal, seeded)
-                f32 = torch.randn(base.features.shape, generator=g, dtype=torch.float32)
-            f = f32.to(device)
+                f = torch.from_numpy(base.features).to(device)
+            else:  # same shape and distribution, different values (standard normal, seeded, drawn on the device)
+                f = torch.randn(base.features.shape, generator=g, dtype=torch.float32, device=device)
             if w.dtype == "bf16":
                 f = f.to(torch.bfloat16)
             self.feats.append(f.contiguous())
@@ -397,16 +404,130 @@ def measure_e2e(torch, w, args, device, steps, warmup, dist_barrier):
             "h2d": frames * (w.feature_bytes + w.matrix_bytes), "d2h": frames * w.output_bytes, "total_ms": total_ms}
 
 
+def measure_capacity(torch, device, base_ms: float, base_mb: float):
+    """Deployment capacity in the manner of the paper's Table 5, on this GPU and at the paper's reference shape: the
+    largest number of height bins and the largest square BEV grid the fused operator handles within the latency of
+    the tensorised baseline (Z = 8, 200 x 200), and the largest grid within the baseline's peak memory."""
+    from paper_2607_10071_b200 import binding as fb
+    wp = wl.get("paper_shape")
+    inp = wl.make_inputs(wp)
+    feats = torch.from_numpy(inp.features).to(device)
+    mats = torch.from_numpy(inp.lidar2img).to(device)
+    cell = (wp.bev_range[1] - wp.bev_range[0]) / wp.grid[0]
+
+    def latency_ms(X, Z):
+        half = X * cell / 2.0
+        rng = (-half, half, -half, half, wp.bev_range[4], wp.bev_range[5])
+        out = torch.empty((wp.B, X, X, wp.C), dtype=torch.float32, device=device)
+        call = lambda: fb.sampling_vt(feats, mats, wp.img_hw, rng, (X, X, Z), wp.reduce, out=out)
+        for _ in range(2):
+            call()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 5
+        a.record()
+        for _ in range(reps):
+            call()
+        b.record()
+        torch.cuda.synchronize()
+        del out
+        return a.elapsed_time(b) / reps
+
+    def largest(fits, lo, hi):
+        """Largest n in [lo, hi] with fits(n), assuming monotonicity and fits(lo)."""
+        while lo < hi:
+            mid = (lo + hi + 1) // 2
+            if fits(mid):
+                lo = mid
+            else:
+                hi = mid - 1
+        return lo
+
+    res = {"budget_latency_ms": base_ms, "budget_memory_mb": base_mb,
+           "grid_rule": "cell size and height range of the paper's shape kept; the grid grows around the ego"}
+    if latency_ms(wp.grid[0], wp.grid[2]) <= base_ms:
+        res["max_height_bins_within_latency"] = largest(lambda z: latency_ms(wp.grid[0], z) <= base_ms, wp.grid[2], 4096)
+        res["max_grid_within_latency"] = largest(lambda x: latency_ms(x, wp.grid[2]) <= base_ms, wp.grid[0], 6000)
+    # memory of the fused operator = its inputs and its output (it has no workspace): solve for the grid
+    budget = base_mb * 1e6 - wp.feature_bytes - wp.matrix_bytes
+    g = int((budget / (wp.C * 4.0)) ** 0.5)
+    ms = latency_ms(g, wp.grid[2])       # and run it once at that size
+    res["max_grid_within_memory"] = g
+    res["latency_ms_at_max_grid_within_memory"] = ms
+    res["paper_rtx_a6000"] = {"max_height_bins_within_latency": 58, "max_grid_within_latency": 529,
+                              "max_grid_within_memory": 1992, "source": "Table 5"}
+    return res
+
+
+def full_block(torch, w, args, device, rank, barrier, steps, warmup, world, reduce_max, kernel=0, tune=(0, 0, 0, 0),
+               clock_sampler=None, cpu_seconds=12.0):
+    """Everything the JSON line carries for one workload: device-resident throughput, roofline, end to end, memory,
+    CPU baseline."""
+    from paper_2607_10071_b200 import binding as fb
+    if clock_sampler is not None and rank == 0:
+        clock_sampler.start()
+    m = measure_workload(torch, w, args, device, rank, barrier, steps, warmup, kernel, tune)
+    clocks = clock_sampler.stop() if (clock_sampler is not None and rank == 0) else None
+    frames = m["frames"]
+    value, total_ms = whole_job_value(m["total_ms"], steps * frames * w.sample_channels, world, reduce_max)
+    launch_ms = statistics.mean(m["per_step_ms"]) / frames  # average duration of one launch (one frame)
+
+    # peak memory of one call: nothing may be allocated
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    torch.cuda.reset_peak_memory_stats()
+    a0 = torch.cuda.max_memory_allocated()
+    fb.flashbev_sampling_vt(m["df"].params[0], torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    workspace = (torch.cuda.max_memory_allocated() - a0) + max(0, free0 - torch.cuda.mem_get_info()[0])
+    m.pop("df")
+    torch.cuda.empty_cache()
+
+    e2e_steps = max(3, steps // 4)
+    e2e = measure_e2e(torch, w, args, device, e2e_steps, 3, barrier)
+    e2e_value, _ = whole_job_value(e2e["total_ms"], e2e_steps * e2e["frames"] * w.sample_channels, world, reduce_max)
+
+    peak, peak_kind = measured_peaks()
+    achieved = w.unique_bytes / (launch_ms * 1e-3) / 1e9
+    blk = {
+        "value": value, "ms_per_step": total_ms / steps, "latency_ms": launch_ms,
+        "latency_ms_median": statistics.median(m["per_step_ms"]) / frames,
+        "latency_ms_min": min(m["per_step_ms"]) / frames,
+        "config": {"workload": w.name, "B": w.B, "N": w.N, "C": w.C, "feat_hw": list(w.feat_hw), "img_hw": list(w.img_hw),
+                   "grid": list(w.grid), "bev_range": list(w.bev_range), "reduce": w.reduce, "frames_per_step": frames,
+                   "l2": "inputs and outputs of a step total %.0f MB (> 3x the 126 MB L2), no flush" % (frames * w.unique_bytes / 1e6),
+                   "launch": "direct" if args.no_graph else "cuda graph replay of the step's launches",
+                   "kernel": m["kernel"]},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": NCU_DRAM_TRAFFIC.get(w.name), "traffic_note": TRAFFIC_NOTE,
+                     "algorithmic_bytes_per_launch": w.unique_bytes, "frac_of_8TBs_nominal": achieved / 8000.0,
+                     "target_frac": 0.5, "target_met": bool(achieved / peak >= 0.5),
+                     "what_binds": "not HBM: a cached gather (features stay in L2); instruction issue and the L1 data "
+                                   "pipe set the time, see profiles/"},
+        "peak_mb": {"workspace_allocated_by_call": workspace / 1e6, "output": w.output_bytes / 1e6,
+                    "inputs_plus_output": w.unique_bytes / 1e6},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "frames_per_step": e2e["frames"],
+                "api": "flashbev_sampling_vt_host (pinned host buffers, frames round-robin over 3 streams)"},
+        "gpu_launches": steps * m["launches_per_step"],
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1 and rank == 0:
+        blk["cpu_baseline"] = oracle_throughput(w, cpu_seconds, 200)
+    return blk
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="representative", choices=list(wl.WORKLOADS))
-    ap.add_argument("--frames", type=int, default=0, help="frames per step (0: enough to exceed 3x L2)")
+    ap.add_argument("--workload", default="long_range", choices=list(wl.WORKLOADS),
+                    help="headline workload (default: the largest configuration by unique bytes and outputs)")
+    ap.add_argument("--frames", type=int, default=0, help="frames per step (0: at least 64, and enough to exceed 3x L2)")
     ap.add_argument("--no-graph", action="store_true", help="time direct launches instead of a CUDA graph replay")
-    ap.add_argument("--no-table", action="store_true", help="skip the per-configuration table")
+    ap.add_argument("--no-table", action="store_true", help="skip the per-configuration table, the second full block and the context")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 per-output, 2 tiled")
     ap.add_argument("--tune", type=str, default="0,0,0,0")
@@ -441,13 +562,7 @@ def main():
             pass
     barrier()
     fb.lib()
-    tune = tuple(int(t) for t in args.tune.split(","))
-
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    m = measure_workload(torch, w, args, device, rank, barrier, args.steps, args.warmup, args.kernel, tune)
-    clocks = sampler.stop() if rank == 0 else None
+    tune = tuple(int(t, 0) for t in args.tune.split(","))
 
     # max over ranks of the device time of the K steps
     def reduce_max(x):
@@ -455,101 +570,96 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    frames = m["frames"]
-    value, total_ms = whole_job_value(m["total_ms"], args.steps * frames * w.sample_channels, world, reduce_max)
-    launch_ms = statistics.mean(m["per_step_ms"]) / frames  # average duration of one launch (one frame)
+    head = full_block(torch, w, args, device, rank, barrier, args.steps, args.warmup, world, reduce_max, args.kernel, tune,
+                      ClockSampler(local_rank))
 
-    # peak memory of one call: nothing may be allocated
-    torch.cuda.synchronize()
-    free0 = torch.cuda.mem_get_info()[0]
-    torch.cuda.reset_peak_memory_stats()
-    a0 = torch.cuda.max_memory_allocated()
-    fb.flashbev_sampling_vt(m["df"].params[0], torch.cuda.current_stream().cuda_stream)
-    torch.cuda.synchronize()
-    workspace = (torch.cuda.max_memory_allocated() - a0) + max(0, free0 - torch.cuda.mem_get_info()[0])
-
-    e2e = measure_e2e(torch, w, args, device, max(3, args.steps // 4), 3, barrier)
-    e2e_value, _ = whole_job_value(e2e["total_ms"], max(3, args.steps // 4) * e2e["frames"] * w.sample_channels,
-                                   world, reduce_max)
-
-    table = {}
+    table, context, second = {}, {}, {}
+    side_steps = max(3, args.steps // 4)
     if not args.no_table and world == 1:
+        # the configuration with the most samples (64 height bins) gets a full block of its own
+        other = "high_res" if w.name != "high_res" else "long_range"
+        second[other] = full_block(torch, wl.get(other), args, device, rank, barrier, side_steps, 3, world, reduce_max,
+                                   cpu_seconds=6.0)
+        from oracle import flashbev_oracle as orc   # (CPU baseline leg: the oracle as it stands, timed beside the GPU)
+        orc.build()
         for name in wl.CONFIG_ORDER:
             wi = wl.get(name)
-            mi = measure_workload(torch, wi, args, device, rank, barrier, max(3, args.steps // 4), 3)
+            mi = measure_workload(torch, wi, args, device, rank, barrier, side_steps, 3)
             extra = measure_regimes(torch, mi.pop("df"), device)
+            torch.cuda.empty_cache()
             lat = statistics.mean(mi["per_step_ms"]) / mi["frames"]
             peak, _ = measured_peaks()
-            table[name] = {"latency_ms": round(lat, 5), "sample_channels_per_s": wi.sample_channels / (lat * 1e-3),
-                           "latency_ms_median": round(statistics.median(mi["per_step_ms"]) / mi["frames"], 5),
-                           "latency_ms_min": round(min(mi["per_step_ms"]) / mi["frames"], 5),
-                           "valid_sample_channels_per_s": extra["valid_samples"] * wi.C / (lat * 1e-3), **extra,
-                           "hbm_roofline_frac_of_measured": wi.unique_bytes / (lat * 1e-3) / 1e9 / peak,
-                           "hbm_roofline_frac_of_8TBs": wi.unique_bytes / (lat * 1e-3) / 1e9 / 8000.0,
-                           "unique_mb": round(wi.unique_bytes / 1e6, 3), "output_mb": round(wi.output_bytes / 1e6, 3),
-                           "kernel": mi["kernel"], "frames_per_step": mi["frames"], "reduce": wi.reduce}
+            row = {"latency_ms": round(lat, 5), "sample_channels_per_s": wi.sample_channels / (lat * 1e-3),
+                   "latency_ms_median": round(statistics.median(mi["per_step_ms"]) / mi["frames"], 5),
+                   "latency_ms_min": round(min(mi["per_step_ms"]) / mi["frames"], 5),
+                   "valid_sample_channels_per_s": extra["valid_samples"] * wi.C / (lat * 1e-3), **extra,
+                   "hbm_roofline_frac_of_measured": wi.unique_bytes / (lat * 1e-3) / 1e9 / peak,
+                   "hbm_roofline_frac_of_8TBs": wi.unique_bytes / (lat * 1e-3) / 1e9 / 8000.0,
+                   "unique_mb": round(wi.unique_bytes / 1e6, 3), "output_mb": round(wi.output_bytes / 1e6, 3),
+                   "kernel": mi["kernel"], "frames_per_step": mi["frames"], "reduce": wi.reduce}
+            if not args.no_cpu_baseline:
+                inp = wl.make_inputs(wi)
+                t0 = time.perf_counter()
+                orc.sampling_vt(inp.features, inp.lidar2img, wi.img_hw, wi.bev_range, wi.grid, wi.reduce)
+                row["cpu_oracle_ms_per_frame"] = (time.perf_counter() - t0) * 1e3
+                row["cpu_oracle_cores"] = orc.max_threads()
+                if name in ("tiny", "representative"):
+                    t0 = time.perf_counter()
+                    orc.sampling_vt(inp.features, inp.lidar2img, wi.img_hw, wi.bev_range, wi.grid, wi.reduce, threads=1)
+                    row["cpu_oracle_one_thread_ms_per_frame"] = (time.perf_counter() - t0) * 1e3
+            if wi.reduce == wl.REDUCE_MEAN_OVER_VALID:
+                # the paper's own normalisation (Eq. 1) on the same shape
+                me = measure_workload(torch, wl.get(name, reduce=wl.REDUCE_CAMERA_MEAN_Z_SUM), args, device, rank, barrier,
+                                      side_steps, 3)
+                me.pop("df")
+                row["latency_ms_eq1_mode"] = round(statistics.mean(me["per_step_ms"]) / me["frames"], 5)
+            table[name] = row
 
-    context = {}
-    if not args.no_table and world == 1:
         # the paper's own reference shape (Sec. 4.1: C=128 fp32, 56x100 maps, 200x200x8, Eq. 1), forward and
         # backward, next to the paper's figures on its hardware -- context, not a target
         wp = wl.get("paper_shape")
-        mf = measure_workload(torch, wp, args, device, rank, barrier, max(3, args.steps // 4), 3)
+        mf = measure_workload(torch, wp, args, device, rank, barrier, side_steps, 3)
         mf.pop("df")
+        torch.cuda.empty_cache()
         context["paper_shape"] = {
             "forward_latency_ms": statistics.mean(mf["per_step_ms"]) / mf["frames"],
-            "backward_latency_ms": measure_backward(torch, wp, args, device, max(3, args.steps // 4), 3, barrier),
+            "backward_latency_ms": measure_backward(torch, wp, args, device, side_steps, 3, barrier),
             "paper_forward_ms": 1.77, "paper_backward_ms": 3.27, "paper_hardware": "RTX A6000, FP32 (Table 4)",
             "paper_trt_forward_ms": 1.128, "paper_trt_hardware": "RTX 4070 Ti SUPER, TensorRT FP32 (Table 6)"}
-        context["paper_shape"]["tensorized_pytorch_baseline_on_this_gpu"] = measure_tensorized(torch, wp, device)
+        tens = measure_tensorized(torch, wp, device)
+        context["paper_shape"]["tensorized_pytorch_baseline_on_this_gpu"] = tens
         context["paper_shape"]["paper_tensorized_forward"] = {"latency_ms": 9.18, "peak_mb": 1971.94,
                                                               "hardware": "RTX A6000 (Table 4)"}
+        if tens:
+            context["paper_shape"]["deployment_capacity"] = measure_capacity(torch, device, tens["latency_ms"], tens["peak_mb"])
         context["representative_tensorized_pytorch_baseline"] = measure_tensorized(torch, wl.get("representative"), device)
         context["flashsca_bevformer_base"] = {
             f"P={P}": dict(measure_sca(torch, device, P), paper_flashsca_ms=ms, paper_bevformer_sca_ms=base,
                            paper_hardware="RTX 4070 Ti SUPER, TensorRT FP32 (Table 7)")
             for P, ms, base in ((8, 5.27, 8.96), (16, 8.16, 15.81), (32, 13.90, 29.27))}
         context["flashsca_bevformer_base"]["P=8, bf16 values"] = measure_sca(torch, device, 8, bf16=True)
-        context["representative_backward_latency_ms"] = measure_backward(
-            torch, w if w.name == "representative" else wl.get("representative"), args, device,
-            max(3, args.steps // 4), 3, barrier)
+        context["representative_backward_latency_ms"] = measure_backward(torch, wl.get("representative"), args, device,
+                                                                          side_steps, 3, barrier)
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peaks()
-    achieved = w.unique_bytes / (launch_ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if w.dtype == "f32" else "bf16 features, f32 accumulate", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "N": w.N, "C": w.C, "feat_hw": list(w.feat_hw), "img_hw": list(w.img_hw),
-                   "grid": list(w.grid), "bev_range": list(w.bev_range), "reduce": w.reduce, "frames_per_step": frames,
-                   "l2": "inputs of a step total %.0f MB (> 3x the 126 MB L2), no flush" % (frames * w.unique_bytes / 1e6),
-                   "launch": "direct" if args.no_graph else "cuda graph replay of the step's launches",
-                   "kernel": m["kernel"]},
-        "latency_ms": launch_ms,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "traffic": NCU_DRAM_TRAFFIC.get(w.name),
-                     "algorithmic_bytes_per_launch": w.unique_bytes,
-                     "frac_of_8TBs_nominal": achieved / 8000.0},
-        "peak_mb": {"workspace_allocated_by_call": workspace / 1e6, "output": w.output_bytes / 1e6,
-                    "inputs_plus_output": w.unique_bytes / 1e6},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                "frames_per_step": e2e["frames"], "api": "flashbev_sampling_vt_host (pinned host buffers, frames round-robin over 3 streams)"},
-        "gpu_launches": args.steps * m["launches_per_step"],
-        "clocks": clocks,
+        "config": head["config"], "latency_ms": head["latency_ms"], "roofline": head["roofline"], "peak_mb": head["peak_mb"],
+        "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],
+        "cpu_baseline": head.get("cpu_baseline"),
     }
+    if second:
+        line["also_measured"] = second
     if table:
         line["configs"] = table
     if context:
         line["context"] = context
-    if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = oracle_throughput(w, 12.0, 200)
-    elif world == 1:
-        line["cpu_baseline"] = None
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

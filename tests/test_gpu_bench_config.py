@@ -11,7 +11,7 @@ from tests import parity
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["representative", "half_taller"])
+@pytest.mark.parametrize("name", ["representative", "half_taller", "long_range"])
 def test_graph_replay_of_a_benchmark_step(oracle, name):
     import torch
     w = wl.get(name)

@@ -118,9 +118,12 @@ typedef struct flashbev_vt_params {
                                   tune[1]: lanes per cell; tune[2]: height bins (or texel rows) per geometry run, rounded
                                   down to a power of two; tune[3]: bits 0-3 warps per CTA (1,2,4,8), bits 4-7 / 8-11
                                   sub-blocks per warp in x / y, bits 12-15 super-blocks per warp, bit 16 never / bit 17
-                                  always use 256-bit feature loads, bits 18-19 super-block order (band height 4,1,2,8),
-                                  bits 20-27 record slots per warp in units of 16.  Values that do not fit fall back to
-                                  the defaults */
+                                  always use 256-bit feature loads, bits 18-19 band height of the super-block order
+                                  (2,1,4,8), bits 20-27 record slots per warp in units of 16, bit 28 visit the bands in
+                                  row order instead of from the middle of the grid outwards, bits 29-31 how many of the
+                                  last super-blocks are handed out one sub-block per warp (0 default; 1..7 = 0, 1/4, 1/2,
+                                  1, 3/2, 2, 3 short tasks per resident warp slot).  Values that do not fit fall back
+                                  to the defaults */
     uint32_t *debug_error_word; /* optional DEVICE word, or NULL.  Only the bounds-checked build of the library
                                   (-DFLASHBEV_DEBUG_BOUNDS) uses it: every shared-memory slot, record offset and
                                   output index the tiled kernel computes is range-checked there; an index out of

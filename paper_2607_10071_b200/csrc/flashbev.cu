@@ -57,6 +57,9 @@ struct KParams {
     float inv_n;                // 1 / N
     int blocks_x, blocks_y;     // super-blocks per batch element
     int band, reps;             // super-block order: bands of `band` rows; super-blocks per warp
+    int nbands, centre_out;     // number of bands; visit them from the middle of the grid outwards
+    int total_sbs;              // super-blocks in visiting order (bands * band * blocks_y)
+    int whole_tasks;            // super-blocks (in visiting order) taken whole by one warp; the rest go one sub-block per warp
     int walk, walk_shift;       // height bins (or texel rows) per run: a power of two, 2 walk <= slots
     int inv_g;                  // ceil(65536 / g)
     int slots;                  // record slots per warp
@@ -806,16 +809,21 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
         return true;
     };
     if (sbx < 1 || sby < 1 || !fits(sbx, sby)) {
+        // (from sweeps) about 10-16 cells per warp -- enough columns to keep the geometry lanes busy -- but fewer if
+        // that leaves the SMs less than three rounds of warps, never more than the record slots hold in one round
+        // (a cell writes roughly 1.2 Z + 12 records on surround rigs) and never fewer warps than the SMs can hold.
         static const int shapes[][2] = {{1, 1}, {1, 2}, {2, 2}, {2, 3}, {2, 4}, {3, 3}, {3, 4}, {4, 4}};
-        // ... at most four sub-blocks, and few enough cells that every SM still gets a full set of warps
-        const long long cells = (long long)p->B * p->X * p->Y;
-        const int want = (int)std::max<long long>(k.cpw, std::min<long long>(std::min<long long>(4 * k.cpw, (long long)(k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0))),
-                                                                          cells / ((long long)sm_count() * 20)));
+        const long long cells = (long long)p->B * p->X * p->Y, warp_slots = (long long)sm_count() * 20;
+        double want = std::min(16.0, std::max(10.0, (double)cells / (3.0 * warp_slots)));
+        want = std::min(want, (double)cells / warp_slots);
+        want = std::min(want, k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0));
         sbx = sby = 1;
+        double best = 1e30;
         for (const auto &sh : shapes) {
             const int ct = sh[0] * sh[1] * k.cpw;
-            if (!fits(sh[0], sh[1]) || ct > want) break;
-            sbx = sh[0], sby = sh[1];
+            if (!fits(sh[0], sh[1])) break;
+            const double miss = ct > want ? ct - want : want - ct;
+            if (miss < best) best = miss, sbx = sh[0], sby = sh[1];
         }
     }
     if (!fits(sbx, sby)) return FLASHBEV_UNSUPPORTED;
@@ -823,17 +831,30 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     k.ct = k.sbn * k.cpw;
     k.blocks_x = (p->X + sbx * k.wx - 1) / (sbx * k.wx);
     k.blocks_y = (p->Y + sby * k.wy - 1) / (sby * k.wy);
-    { const int bc = (p->tune[3] >> 18) & 3; k.band = bc == 1 ? 1 : (bc == 2 ? 2 : (bc == 3 ? 8 : 4)); }
+    { const int bc = (p->tune[3] >> 18) & 3; k.band = bc == 1 ? 1 : (bc == 2 ? 4 : (bc == 3 ? 8 : 2)); }
     k.reps = (p->tune[3] >> 12) & 0xf;
     if (k.reps < 1) k.reps = 1;
     k.wcap = k.colcap * runs;
     k.den_bytes = eq1 ? (int)align16((size_t)k.ct * p->Z) : 0;
 
     const long long bands = (k.blocks_x + k.band - 1) / k.band;
-    const long long ids = bands * k.band * k.blocks_y;
+    k.nbands = (int)bands;
+    k.centre_out = !((p->tune[3] >> 28) & 1);
+    const long long sbs = bands * k.band * k.blocks_y;  // super-blocks in visiting order (those past the grid's edge do nothing)
+    // the tail of the order is split into single sub-blocks: about one warp's worth per resident warp slot
+    // (0 = default: one short task per resident warp slot when a super-block has four or more sub-blocks)
+    static const double tail_factor[8] = {-1.0, 0.0, 0.25, 0.5, 1.0, 1.5, 2.0, 3.0};
+    double tf = tail_factor[((unsigned)p->tune[3] >> 29) & 7];
+    if (tf < 0.0) tf = k.sbn >= 4 ? 1.0 : 0.0;
+    long long tail = k.sbn > 1 ? std::min<long long>(sbs, (long long)(sm_count() * 20 * tf) / k.sbn) : 0;
+    if (k.reps > 1) tail = 0;
+    k.total_sbs = (int)sbs;
+    k.whole_tasks = (int)(sbs - tail);
+    const long long ids = (sbs - tail) + tail * k.sbn;
     const long long ctas = (ids + (long long)warps * k.reps - 1) / ((long long)warps * k.reps);
     const int cblocks = (k.vecs + g * V - 1) / (g * V);
-    if (ctas > 2147483647LL || cblocks > 65535 || p->B > 65535) return FLASHBEV_UNSUPPORTED;
+    if (ctas > 2147483647LL || ids + (long long)warps * k.reps >= 2147483647LL || cblocks > 65535 || p->B > 65535)
+        return FLASHBEV_UNSUPPORTED;  // (task ids are 32-bit in the kernel)
     grid = dim3((unsigned)ctas, (unsigned)cblocks, (unsigned)p->B);
     // adjacent vectors and 256-bit loads: half the load instructions (bf16 features are issue-bound), and whole
     // texels per cell where the strided 16-byte segments of a cell would not cover whole 128-byte lines

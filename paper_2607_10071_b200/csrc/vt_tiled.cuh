@@ -767,17 +767,30 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
 
     for (int rep = 0; rep < p.reps; ++rep) {
         // ---- which super-block: ids run along y inside bands of `band` rows of super-blocks
-        const int id = (blockIdx.x * WARPS + warp) * p.reps + rep;
+        int id = (blockIdx.x * WARPS + warp) * p.reps + rep;
+        // The last super-blocks of the order are handed out one sub-block per warp: short tasks for the end of the
+        // grid, when the SMs run out of work one warp at a time.
+        int s_begin = 0, s_end = p.sbn;
+        if (id >= p.whole_tasks) {
+            const int k = id - p.whole_tasks, q = k / p.sbn;
+            id = p.whole_tasks + q, s_begin = k - q * p.sbn, s_end = s_begin + 1;
+        }
+        if (id >= p.total_sbs) continue;  // (padding warps of the last CTA; warp-uniform)
         const int per_band = p.band * p.blocks_y;
-        const int bandi = id / per_band, rem = id - bandi * per_band;
+        int bandi = id / per_band;
+        const int rem = id - bandi * per_band;
+        if (p.centre_out) {  // bands from the middle of the grid outwards: the cells around the ego write the most records
+            const int half = (bandi + 1) >> 1;
+            bandi = ((p.nbands - 1) >> 1) + ((bandi & 1) ? half : -half);
+        }
         const int by = rem / p.band, bx = bandi * p.band + (rem - by * p.band);
-        if (bx >= p.blocks_x) continue;  // warp-uniform
+        if ((unsigned)bx >= (unsigned)p.blocks_x || (unsigned)by >= (unsigned)p.blocks_y) continue;  // past the grid's edge; warp-uniform
         const int ix0 = bx * (p.sbx * p.wx), iy0 = by * (p.sby * p.wy);
 
         unsigned in_mask;  // bit c: cell c of the super-block is inside the grid
         {
             const int lx = my_tab & 0xff, ly = my_tab >> 8;
-            const bool in = (lane < p.ct) && (ix0 + lx < p.X) && (iy0 + ly < p.Y);
+            const bool in = (lane >= s_begin * p.cpw) && (lane < s_end * p.cpw) && (ix0 + lx < p.X) && (iy0 + ly < p.Y);
             const double nan = __longlong_as_double(0x7ff8000000000000LL);
             if (lane < p.ct)
                 sm.cellxy[lane] = make_double2(in ? p.x_min + ((double)(ix0 + lx) + 0.5) * p.dx : nan,
@@ -788,10 +801,10 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
         survey_candidates(p, cx, in_mask);
 
         // ---- segments: as many sub-blocks as have at most `colcap` surviving columns together (normally all of them)
-        for (int s0 = 0; s0 < p.sbn;) {
+        for (int s0 = s_begin; s0 < s_end;) {
             const int jb = sm.cfirst[s0 * p.cpw];
             int s1 = s0 + 1;
-            while (s1 < p.sbn && sm.cfirst[min((s1 + 1) * p.cpw, p.ct)] - jb <= p.colcap) ++s1;
+            while (s1 < s_end && sm.cfirst[min((s1 + 1) * p.cpw, p.ct)] - jb <= p.colcap) ++s1;
             const int ncols = sm.cfirst[min(s1 * p.cpw, p.ct)] - jb;  // <= colcap: a sub-block has at most cpw * N candidates
             const int nw = build_columns(p, cx, jb, ncols, s0 * p.cpw, min(s1 * p.cpw, p.ct));
 

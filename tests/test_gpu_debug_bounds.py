@@ -75,6 +75,23 @@ def test_many_rounds_and_odd_shapes_make_no_out_of_range_index(oracle, checked):
         assert cnt.min() >= 0
 
 
+@pytest.mark.parametrize("name", ["half_taller", "paper_shape", "representative"])
+def test_launch_geometry_hints_make_no_out_of_range_index(oracle, checked, name):
+    """Super-block shapes, tail lengths, orders and warps per CTA that leave padding warps in the last CTA and
+    partial super-blocks at the grid's edge."""
+    inp = wl.make_inputs(wl.get(name))
+    w = inp.workload
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, w.reduce)
+    shapes = [0, (1 << 4) | (2 << 8), (2 << 4) | (3 << 8), (3 << 4) | (3 << 8)]
+    for shape in shapes:
+        for tail in range(8):
+            for extra in (0, 1 << 28, 2, 8, 1 << 18):       # default, row-major order, 2 / 8 warps per CTA, single-row bands
+                tune = (0, 0, 0, shape | (32 << 20) | (tail << 29) | extra)
+                out, cnt, violations = run_checked(checked, inp, w.reduce, tune)
+                assert violations == 0, f"{name} tune[3]={tune[3]:#x}: {violations} out-of-range indices"
+                assert np.array_equal(cnt[ref.flagged == 0], ref.count[ref.flagged == 0]), hex(tune[3])
+
+
 def test_backward_makes_no_out_of_range_index(checked):
     """The backward entry point has no error-word field: run it in the checked build for its clamping only and
     compare with the normal build (the scatter order differs from run to run, hence a tolerance)."""

@@ -391,7 +391,7 @@ __device__ __forceinline__ int affine_run_records(const ColDesc &D, int len) { r
 // ---- step 2: walker of an affine column.  Writes exactly affine_run_records() records. -------------------------
 // A run of rows [ra, rb) takes the bins whose upper tap lies in rows ra - 1 .. rb - 1: a row's weight is the (1 - ty)
 // of the bins in it plus the ty of the bins in the row above, so every run is complete by itself and neighbouring
-// runs share no record.  The run's own record slots serve as the accumulators of its rows.
+// runs share no record.  Bins are taken in order and a row's record is written when the bins have moved past it.
 __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm, const ColDesc &D, int u0, int len,
                                             int *out_off, float2 *out_w, int cap)
 {
@@ -427,13 +427,18 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
             return k;
         };
         const int kb = first_bin_at((double)(ra - 1)), ke = first_bin_at((double)(ra + len));
-        float *w = reinterpret_cast<float *>(out_w);  // w[2 i]: weight of row ra + i
-        for (int i = 0; i < len; ++i) w[2 * i] = 0.f;
+        // The two rows the current bin touches are kept in registers; a row is written, once, when the bins have
+        // left it (its weight is complete then: the (1 - ty) of its own bins and the ty of the bins of the row above).
+        int off = FB_IDX(offc + ra * rowv, p.nvec_cam - p.vecs - p.rstep + 1 - (len - 1) * rowv, p.err) - rowv;
+        int icur = -1;  // a0: weight of row icur, a1: of row icur + 1 (relative to ra); pw, po, off belong to row icur
+        float a0 = 0.f, a1 = 0.f;
+        float2 *pw = out_w - 1;
+        int *po = out_off - 1;
         double kd = (double)kb;
         const unsigned char *dk = den + kb * dstep;
         for (int k = kb; k < ke; ++k, kd += 1.0, dk += dstep) {
             const double fy = fma(kd, S, A), fl = floor(fy);
-            const int i = (int)fl - ra;  // row of the upper tap, relative
+            const int i = (int)fl - ra;  // row of the upper tap, relative: -1 .. len - 1, never decreasing
             float ty = (float)(fy - fl), tu = 1.f - ty;
             if (eq1) {
 #ifdef FLASHBEV_DEBUG_BOUNDS
@@ -442,15 +447,20 @@ __device__ __forceinline__ void walk_affine(const KParams &p, const WarpSmem &sm
                 const float sc = 1.f / (float)max(1, (int)*dk);
                 ty *= sc, tu *= sc;
             }
-            if ((unsigned)i < (unsigned)len) w[2 * i] += tu;
-            if ((unsigned)(i + 1) < (unsigned)len) w[2 * i + 2] += ty;
+            if (i != icur) {
+                if ((unsigned)icur < (unsigned)len) *pw = make_float2(cl * a0, cr * a0), *po = off;
+                a0 = a1, a1 = 0.f, ++icur, ++pw, ++po, off += rowv;
+                while (i != icur && icur < len) {  // a row without a bin of its own (steps of more than one row per bin)
+                    *pw = make_float2(cl * a0, cr * a0), *po = off;
+                    a0 = 0.f, ++icur, ++pw, ++po, off += rowv;
+                }
+            }
+            a0 += tu, a1 += ty;
         }
-        int off = FB_IDX(offc + ra * rowv, p.nvec_cam - p.vecs - p.rstep + 1 - (len - 1) * rowv, p.err);
-        for (int i = 0; i < len; ++i, off += rowv) {
-            const float wi = w[2 * i];
-            out_w[i] = make_float2(cl * wi, cr * wi);
-            out_off[i] = off;
-        }
+        if ((unsigned)icur < (unsigned)len) *pw = make_float2(cl * a0, cr * a0), *po = off;
+        a0 = a1;
+        for (++icur, ++pw, ++po, off += rowv; icur < len; ++icur, ++pw, ++po, off += rowv, a0 = 0.f)
+            *pw = make_float2(cl * a0, cr * a0), *po = off;
     } else {
         // rows of successive bins never coincide: two records per bin (a row outside the map: weight 0, clamped)
         len = min(len, cap / 2);

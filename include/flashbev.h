@@ -212,6 +212,8 @@ typedef struct flashbev_vt_backward_params {
     int32_t reduce;            /* flashbev_reduce */
     float *grad_features;      /* device, [B][N][feat_h][feat_w][C] float32; overwritten */
     int32_t tune[4];           /* as in flashbev_vt_params; 0 = defaults */
+    uint32_t *debug_error_word; /* as in flashbev_vt_params (bounds-checked build only); callers built against a
+                                  header without this field are accepted */
 } flashbev_vt_backward_params;
 
 flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params *p, void *stream);

@@ -63,6 +63,7 @@ class VtBackwardParams(ctypes.Structure):
         ("reduce", ctypes.c_int32),
         ("grad_features", ctypes.c_void_p),
         ("tune", ctypes.c_int32 * 4),
+        ("debug_error_word", ctypes.c_void_p),
     ]
 
 
@@ -235,7 +236,7 @@ def flashbev_sampling_vt_multires(base: VtParams, feature_ptrs, feat_hws, stream
 
 
 def make_backward_params(grad_out_ptr, lidar2img_ptr, B, N, C, feat_hw, img_hw, bev_range, grid, reduce,
-                         grad_features_ptr, tune=(0, 0, 0, 0)) -> VtBackwardParams:
+                         grad_features_ptr, tune=(0, 0, 0, 0), debug_error_word=None) -> VtBackwardParams:
     p = VtBackwardParams()
     p.struct_size = ctypes.sizeof(VtBackwardParams)
     p.grad_out, p.lidar2img, p.grad_features = grad_out_ptr, lidar2img_ptr, grad_features_ptr
@@ -247,6 +248,7 @@ def make_backward_params(grad_out_ptr, lidar2img_ptr, B, N, C, feat_hw, img_hw, 
     p.reduce = reduce
     for i, t in enumerate(tune):
         p.tune[i] = int(t)
+    p.debug_error_word = debug_error_word
     return p
 
 

@@ -991,7 +991,7 @@ flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_s
 // ---- backward --------------------------------------------------------------------------------
 flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params *q, void *stream_)
 {
-    if (!q || q->struct_size < sizeof(flashbev_vt_backward_params)) return FLASHBEV_INVALID_ARG;
+    if (!q || q->struct_size < offsetof(flashbev_vt_backward_params, debug_error_word)) return FLASHBEV_INVALID_ARG;
     if (!q->grad_out || !q->grad_features) return FLASHBEV_INVALID_ARG;
     // same geometry description as the forward: validate it through the forward's checks
     flashbev_vt_params p = {};
@@ -1007,6 +1007,7 @@ flashbev_status flashbev_sampling_vt_backward(const flashbev_vt_backward_params 
     p.out_dtype = FLASHBEV_F32;
     p.kernel = FLASHBEV_KERNEL_TILED;
     for (int i = 0; i < 4; ++i) p.tune[i] = q->tune[i];
+    p.debug_error_word = q->struct_size >= sizeof(flashbev_vt_backward_params) ? q->debug_error_word : nullptr;
     flashbev_status st;
     if (!params_ok(&p, st)) return st;
     if (((uintptr_t)q->grad_out % 16) || ((uintptr_t)q->grad_features % 16) || ((uintptr_t)q->lidar2img % 4))

@@ -92,20 +92,27 @@ def test_launch_geometry_hints_make_no_out_of_range_index(oracle, checked, name)
                 assert np.array_equal(cnt[ref.flagged == 0], ref.count[ref.flagged == 0]), hex(tune[3])
 
 
-def test_backward_makes_no_out_of_range_index(checked):
-    """The backward entry point has no error-word field: run it in the checked build for its clamping only and
-    compare with the normal build (the scatter order differs from run to run, hence a tolerance)."""
+@pytest.mark.parametrize("name,C,reduce,tune3", [
+    ("tiny", 32, 2, 0), ("tiny", 32, 1, 0), ("representative", 80, 0, 0), ("representative", 24, 2, 0),
+    ("representative", 144, 1, 0), ("representative", 80, 0, (2 << 4) | (4 << 8)),
+])
+def test_backward_makes_no_out_of_range_index(checked, name, C, reduce, tune3):
+    """The backward in the checked build: the error word stays 0 and the result equals the normal build's up to the
+    order of the atomic sums."""
     import torch
-    w = wl.get("tiny")
+    w = wl.get(name, C=C)
     inp = wl.make_inputs(w)
     dev = torch.device("cuda:0")
     X, Y, Z = w.grid
     go = torch.randn((w.B, X, Y, w.C), generator=torch.Generator().manual_seed(3)).to(dev)
     mats = torch.from_numpy(inp.lidar2img).to(dev)
-    ref = fb.sampling_vt_backward(go, mats, w.feat_hw, w.img_hw, w.bev_range, w.grid, 2)
+    ref = fb.sampling_vt_backward(go, mats, w.feat_hw, w.img_hw, w.bev_range, w.grid, reduce)
     gf = torch.empty_like(ref)
-    p = fb.make_backward_params(go.data_ptr(), mats.data_ptr(), w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid, 2,
-                                gf.data_ptr())
+    word = torch.zeros(1, dtype=torch.int32, device=dev)
+    p = fb.make_backward_params(go.data_ptr(), mats.data_ptr(), w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid, reduce,
+                                gf.data_ptr(), (0, 0, 0, tune3), debug_error_word=word.data_ptr())
     fb.flashbev_sampling_vt_backward(p, torch.cuda.current_stream().cuda_stream, library=checked)
     torch.cuda.synchronize()
-    assert torch.allclose(gf, ref, rtol=1e-5, atol=1e-5)
+    assert int(word.item()) == 0
+    scale = float(ref.abs().max())
+    assert float((gf - ref).abs().max()) <= 1e-5 * max(1.0, scale)

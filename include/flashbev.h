@@ -131,18 +131,28 @@ typedef struct flashbev_vt_params {
                                   dereferenced.  The caller zeroes the word before the call and reads it after
                                   synchronising.  The normal build ignores it.  Callers built against an older
                                   header (struct_size without this field) are accepted. */
+    void *workspace;           /* optional DEVICE scratch, 16-byte aligned, or NULL.  Only channel-planar (NCHW)
+                                  tensors use it: with flashbev_workspace_bytes(p) bytes here the features are
+                                  first transposed into it (channels last) and the tiled kernel runs on the copy,
+                                  writing the NCHW output directly; without it NCHW tensors take the generic
+                                  per-output kernel (an order of magnitude slower).  Callers built against a
+                                  header without these two fields are accepted. */
+    size_t workspace_bytes;    /* size of `workspace` */
 } flashbev_vt_params;
 
 /*
  * The operator (Eq. 1; Algorithm 2).  Validates `p` on the host (no CUDA call is made and no
  * device memory is touched when validation fails), then enqueues exactly one kernel on `stream`
- * (a cudaStream_t, passed as void*; NULL = the default stream) and returns without waiting.
- * Uses no device memory beyond `features`, `lidar2img`, `out` and `valid_count_out`.
+ * (two for NCHW tensors with a workspace: a transposing copy first) and returns without waiting
+ * (`stream` is a cudaStream_t, passed as void*; NULL = the default stream).
+ * Uses no device memory beyond `features`, `lidar2img`, `out`, `valid_count_out` and `workspace`.
  */
 flashbev_status flashbev_sampling_vt(const flashbev_vt_params *p, void *stream);
 
-/* Device scratch the operator needs beyond its inputs and outputs: always 0 (Sec. 3.3.1: all
- * intermediates live in registers / on chip).  Exists so callers can assert the contract. */
+/* Device scratch the operator can use beyond its inputs and outputs.  0 for channels-last (NHWC)
+ * tensors (Sec. 3.3.1: all intermediates live in registers / on chip).  For NCHW tensors whose
+ * channel rows are whole 16-byte vectors: the size of a channels-last copy of the features, which
+ * `workspace` may lend to the call (optional; see the field). */
 size_t flashbev_workspace_bytes(const flashbev_vt_params *p);
 
 /*

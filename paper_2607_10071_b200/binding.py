@@ -44,6 +44,8 @@ class VtParams(ctypes.Structure):
         ("valid_count_out", ctypes.c_void_p),
         ("tune", ctypes.c_int32 * 4),
         ("debug_error_word", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
     ]
 
 
@@ -168,7 +170,7 @@ def version() -> int:
 
 def make_params(features_ptr, feat_dtype, lidar2img_ptr, B, N, C, feat_hw, img_hw, bev_range, grid,
                 reduce, out_ptr, valid_count_ptr=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0),
-                layout=NHWC, out_dtype=F32, debug_error_word=None) -> VtParams:
+                layout=NHWC, out_dtype=F32, debug_error_word=None, workspace=None, workspace_bytes=0) -> VtParams:
     p = VtParams()
     p.struct_size = ctypes.sizeof(VtParams)
     p.features, p.feat_dtype, p.layout = features_ptr, feat_dtype, layout
@@ -182,6 +184,7 @@ def make_params(features_ptr, feat_dtype, lidar2img_ptr, B, N, C, feat_hw, img_h
     p.out, p.out_dtype, p.kernel = out_ptr, out_dtype, kernel
     p.valid_count_out = valid_count_ptr
     p.debug_error_word = debug_error_word
+    p.workspace, p.workspace_bytes = workspace, int(workspace_bytes)
     for i, t in enumerate(tune):
         p.tune[i] = int(t)
     return p
@@ -347,10 +350,12 @@ def flashbev_last_kernel_name() -> str:
 
 def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM, out=None,
                 valid_count=None, kernel=KERNEL_AUTO, tune=(0, 0, 0, 0), stream=None, layout=NHWC,
-                out_dtype=F32):
+                out_dtype=F32, workspace=True):
     """features: CUDA tensor [B,N,Hf,Wf,C] (NHWC) or [B,N,C,Hf,Wf] (NCHW), float32 or bfloat16,
     contiguous; lidar2img: CUDA float32 [B,N,4,4].  Returns the output tensor [B,X,Y,C] (NHWC) or
-    [B,C,X,Y] (NCHW), float32 or bfloat16 per ``out_dtype`` (allocated by torch if ``out`` is None)."""
+    [B,C,X,Y] (NCHW), float32 or bfloat16 per ``out_dtype`` (allocated by torch if ``out`` is None).
+    ``workspace``: for NCHW tensors, lend the call the scratch ``flashbev_workspace_bytes`` asks for (a torch
+    allocation, or a uint8 CUDA tensor of the caller's); False: none, the generic kernel runs."""
     import torch
 
     if not features.is_cuda or not lidar2img.is_cuda:
@@ -376,6 +381,11 @@ def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM,
     p = make_params(features.data_ptr(), dt, lidar2img.data_ptr(), B, N, C, (Hf, Wf), img_hw, bev_range,
                     (X, Y, Z), reduce, out.data_ptr(),
                     None if valid_count is None else valid_count.data_ptr(), kernel, tune, layout, out_dtype)
+    if layout == NCHW and workspace is not False and workspace is not None:
+        need = flashbev_workspace_bytes(p)
+        if need:
+            ws = workspace if workspace is not True else torch.empty(need, dtype=torch.uint8, device=features.device)
+            p.workspace, p.workspace_bytes = ws.data_ptr(), ws.numel() * ws.element_size()
     if stream is None:
         stream = torch.cuda.current_stream(features.device).cuda_stream
     with torch.cuda.device(features.device):

@@ -44,6 +44,7 @@ struct KParams {
     float *gfeat;               // backward: gradient of the features [B][N][Hf][Wf][C], fp32, pre-zeroed
     int B, N, C, Hf, Wf, X, Y, Z, reduce;
     int out_bf16;               // store the output as bfloat16 (round to nearest even) instead of float32
+    int out_nchw;               // tiled kernel: the output is [B][C][X][Y] (scalar stores), features are a channels-last copy
     int accumulate;             // add the result to the fp32 output instead of overwriting it (multi-resolution levels)
     double sx, sy;              // image px -> feature px
     double x_min, dx, y_min, dy, z_min, dz;
@@ -570,6 +571,26 @@ __global__ void __launch_bounds__(128, V <= 2 ? 5 : 3) sca_kernel(const ScaParam
 }
 
 // ------------------------------------------------------------------------------------------
+// Channel-planar features [planes][C][HW] -> channels last [planes][HW][C] (T: 2- or 4-byte elements), through a
+// padded shared-memory tile: reads run along HW, writes along C.
+template <typename T>
+__global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const T *__restrict__ in, T *__restrict__ out, int C, int HW)
+{
+    __shared__ T tile[32][33];
+    const size_t plane = (size_t)blockIdx.z * C * HW;
+    const int hw0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int c = c0 + j, hw = hw0 + threadIdx.x;
+        if (c < C && hw < HW) tile[j][threadIdx.x] = in[plane + (size_t)c * HW + hw];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int hw = hw0 + j, c = c0 + threadIdx.x;
+        if (c < C && hw < HW) out[plane + (size_t)hw * C + c] = tile[threadIdx.x][j];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // host side
 
 thread_local int t_last_launches = 0;
@@ -608,7 +629,6 @@ bool params_ok(const flashbev_vt_params *p, flashbev_status &st)
     if (p->out_dtype != FLASHBEV_F32 && p->out_dtype != FLASHBEV_BF16) return false;
     if (p->kernel < 0 || p->kernel > 2) return false;
     st = FLASHBEV_UNSUPPORTED;
-    if (p->layout == FLASHBEV_NCHW && p->kernel == FLASHBEV_KERNEL_TILED) return false;  // planar: per-output kernel only
     if (p->N > kMaxCams) return false;
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
     const double cam_bytes = (double)p->N * p->feat_h * p->feat_w * p->C * (double)elem;
@@ -705,16 +725,38 @@ int sm_count()
     return n;
 }
 
-bool tiled_applicable(const flashbev_vt_params *p)
+// Shapes the tiled kernel serves (whatever the layout): channel rows of whole 16-byte vectors, bounded Z and map size.
+bool tiled_shape_ok(const flashbev_vt_params *p)
 {
-    if (p->layout != FLASHBEV_NHWC) return false;
     const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
     if (((size_t)p->C * elem) % 16) return false;
-    if (((uintptr_t)p->features % 16) || ((uintptr_t)p->out % 16)) return false;
     if (p->Z > 32767) return false;  // a column's interval of height bins is kept in two 16-bit fields
     if (p->reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM && p->Z > 16384) return false;  // per-height camera counts on chip
     const double vecs_total = (double)p->N * p->feat_h * p->feat_w * (double)((size_t)p->C * elem / 16);
     return vecs_total < 2147483648.0;
+}
+
+bool tiled_applicable(const flashbev_vt_params *p)
+{
+    if (p->layout != FLASHBEV_NHWC) return false;
+    if (((uintptr_t)p->features % 16) || ((uintptr_t)p->out % 16)) return false;
+    return tiled_shape_ok(p);
+}
+
+// Bytes of the channels-last copy of NCHW features (0: the shape cannot take the tiled kernel).
+size_t nchw_copy_bytes(const flashbev_vt_params *p)
+{
+    if (p->layout != FLASHBEV_NCHW || !tiled_shape_ok(p)) return 0;
+    return (size_t)p->B * p->N * p->feat_h * p->feat_w * p->C * (p->feat_dtype == FLASHBEV_F32 ? 4 : 2);
+}
+
+// NCHW tensors with a workspace that holds the channels-last copy: transposing copy, then the tiled kernel.
+bool nchw_tiled_applicable(const flashbev_vt_params *p)
+{
+    if (p->struct_size < sizeof(flashbev_vt_params) || !p->workspace) return false;
+    const size_t need = nchw_copy_bytes(p);
+    return need && p->workspace_bytes >= need && (uintptr_t)p->workspace % 16 == 0 &&
+           (long long)p->B * p->N <= 65535 && (p->C + 31) / 32 <= 65535;
 }
 
 template <int V, bool BF16, int WARPS, bool BWD, bool WIDE = false>
@@ -866,7 +908,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     return FLASHBEV_OK;
 }
 
-flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false)
+flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false, bool out_nchw = false)
 {
     KParams k;
     int V, warps;
@@ -874,6 +916,7 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, b
     size_t smem;
     const flashbev_status st = configure_tiled(p, k, V, warps, grid, smem, accumulate);
     if (st != FLASHBEV_OK) return st;
+    k.out_nchw = out_nchw;
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     cudaError_t e;
     static const char *const names[2][3] = {{"tiled_f32_v1", "tiled_f32_v2", "tiled_f32_v4"},
@@ -891,9 +934,54 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, b
     return e == cudaSuccess ? FLASHBEV_OK : FLASHBEV_CUDA_ERROR;
 }
 
+// NCHW tensors on the tiled kernel: features -> channels-last copy in the workspace, output written planar.
+flashbev_status launch_nchw_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate)
+{
+    flashbev_vt_params q = *p;
+    q.features = p->workspace;
+    q.layout = FLASHBEV_NHWC;
+    {   // configure first: nothing is enqueued for a shape the tiled kernel cannot take
+        KParams k;
+        int V, warps;
+        dim3 grid;
+        size_t smem;
+        const flashbev_status st = configure_tiled(&q, k, V, warps, grid, smem, accumulate);
+        if (st != FLASHBEV_OK) return st;
+    }
+    const int HW = p->feat_h * p->feat_w;
+    const dim3 grid((unsigned)((HW + 31) / 32), (unsigned)((p->C + 31) / 32), (unsigned)(p->B * p->N)), block(32, 8);
+    if (p->feat_dtype == FLASHBEV_BF16)
+        nchw_to_nhwc_kernel<uint16_t><<<grid, block, 0, stream>>>(static_cast<const uint16_t *>(p->features),
+                                                                  static_cast<uint16_t *>(p->workspace), p->C, HW);
+    else
+        nchw_to_nhwc_kernel<float><<<grid, block, 0, stream>>>(static_cast<const float *>(p->features),
+                                                               static_cast<float *>(p->workspace), p->C, HW);
+    if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+    const flashbev_status st = launch_tiled(&q, stream, accumulate, true);
+    if (st == FLASHBEV_OK) t_last_kernel = p->feat_dtype == FLASHBEV_BF16 ? "tiled_bf16_nchw" : "tiled_f32_nchw";
+    return st;
+}
+
 flashbev_status run_device(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false)
 {
     flashbev_status st;
+    if (p->layout == FLASHBEV_NCHW) {
+        const bool can = nchw_tiled_applicable(p);
+        if (p->kernel == FLASHBEV_KERNEL_TILED && !can) return FLASHBEV_UNSUPPORTED;
+        if (can && p->kernel != FLASHBEV_KERNEL_PER_OUTPUT) {
+            st = launch_nchw_tiled(p, stream, accumulate);
+            if (st == FLASHBEV_OK) {
+                if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+                t_last_launches = 2;
+                return FLASHBEV_OK;
+            }
+            if (!(st == FLASHBEV_UNSUPPORTED && p->kernel == FLASHBEV_KERNEL_AUTO)) return st;
+        }
+        if ((st = launch_per_output(p, stream, accumulate)) != FLASHBEV_OK) return st;
+        if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+        t_last_launches = 1;
+        return FLASHBEV_OK;
+    }
     const bool tiled = p->kernel == FLASHBEV_KERNEL_TILED || (p->kernel == FLASHBEV_KERNEL_AUTO && tiled_applicable(p));
     if (tiled && !tiled_applicable(p)) return FLASHBEV_UNSUPPORTED;
     st = tiled ? launch_tiled(p, stream, accumulate) : launch_per_output(p, stream, accumulate);
@@ -939,8 +1027,9 @@ flashbev_status flashbev_sampling_vt(const flashbev_vt_params *p, void *stream)
 
 size_t flashbev_workspace_bytes(const flashbev_vt_params *p)
 {
-    (void)p;
-    return 0;
+    flashbev_status st;
+    if (!params_ok(p, st)) return 0;
+    return nchw_copy_bytes(p);
 }
 
 size_t flashbev_host_staging_bytes(const flashbev_vt_params *p)

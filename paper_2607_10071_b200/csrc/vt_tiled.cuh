@@ -919,7 +919,31 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                             for (int e = 0; e < PV; ++e) acc[v][e].x *= gn, acc[v][e].y *= gn;
                     }
                     float *o = p.out + ocell * p.C + out_lane;  // this lane's first channel of the cell
-                    if (!(p.accumulate | p.out_bf16)) {
+                    if (p.out_nchw) {
+                        // channel-planar output [B][C][X][Y]: one scalar per channel, the cells of a sub-block adjacent in y
+                        const size_t plane = (size_t)p.X * p.Y;
+                        const size_t at = ocell + (size_t)b * plane * (size_t)(p.C - 1);  // b C plane + (cell inside the batch element)
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (von[v]) {
+#pragma unroll
+                                for (int e = 0; e < PV; ++e) {
+#pragma unroll
+                                    for (int hl = 0; hl < 2; ++hl) {
+                                        const size_t idx = at + (size_t)(out_lane + v * vstride + e * 2 + hl) * plane;
+                                        float val = hl ? acc[v][e].y : acc[v][e].x;
+                                        if (p.out_bf16) {
+                                            uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + idx;
+                                            if (p.accumulate) val += __bfloat162float(__ushort_as_bfloat16(*ob));
+                                            *ob = __bfloat16_as_ushort(__float2bfloat16_rn(val));
+                                        } else {
+                                            if (p.accumulate) val += p.out[idx];
+                                            __stcs(p.out + idx, val);
+                                        }
+                                    }
+                                }
+                            }
+                    } else if (!(p.accumulate | p.out_bf16)) {
 #pragma unroll
                         for (int v = 0; v < V; ++v)
                             if (von[v]) {

@@ -81,7 +81,7 @@ def good_params(**over):
     (dict(bev_range=(-25, float("inf"), -25, 25, -3, 1)), fb.INVALID_ARG),
     (dict(reduce=3), fb.INVALID_ARG), (dict(feat_dtype=2), fb.INVALID_ARG), (dict(kernel=9), fb.INVALID_ARG),
     (dict(layout=7), fb.INVALID_ARG),
-    (dict(layout=fb.NCHW, kernel=fb.KERNEL_TILED), fb.UNSUPPORTED),  # planar tensors: per-output kernel only
+    (dict(layout=fb.NCHW, kernel=fb.KERNEL_TILED), fb.UNSUPPORTED),  # planar tensors on the tiled kernel need a workspace
     (dict(out_dtype=fb.BF16, out_ptr=16385), fb.MISALIGNED),
     (dict(N=65), fb.UNSUPPORTED),
     (dict(B=1 << 20, grid=(1 << 10, 1 << 10, 4)), fb.UNSUPPORTED),
@@ -114,6 +114,19 @@ def test_host_entry_validates_staging():
     assert fb.flashbev_sampling_vt_host(p, 4096 + 8, need, None, check=False) == fb.MISALIGNED
     assert fb.flashbev_sampling_vt_host(p, 4096, need - 1, None, check=False) == fb.TOO_SMALL
     assert fb.flashbev_workspace_bytes(p) == 0
+
+
+def test_workspace_is_asked_for_planar_tensors_only():
+    """Channels-last tensors need no scratch; NCHW tensors may lend the size of a channels-last copy of the features
+    (only when the channel rows are whole 16-byte vectors: other shapes take the generic kernel anyway)."""
+    assert fb.flashbev_workspace_bytes(good_params()) == 0
+    assert fb.flashbev_workspace_bytes(good_params(layout=fb.NCHW)) == 1 * 6 * 16 * 44 * 32 * 4
+    assert fb.flashbev_workspace_bytes(good_params(layout=fb.NCHW, C=30)) == 0
+    # a workspace that is too small or misaligned is not used: forcing the tiled kernel is refused on the host
+    for ws, nbytes in ((8192, 100), (8200, 1 << 30)):
+        p = good_params(layout=fb.NCHW, kernel=fb.KERNEL_TILED)
+        p.workspace, p.workspace_bytes = ws, nbytes
+        assert fb.flashbev_sampling_vt(p, None, check=False) == fb.UNSUPPORTED
 
 
 def test_multires_arguments_are_validated_on_the_host():

@@ -29,7 +29,7 @@ def _bf16_to_f32(t):
 
 
 @pytest.mark.parametrize("reduce", [SUM, MEAN, EQ1])
-@pytest.mark.parametrize("dtype,C", [("f32", 5), ("f32", 32), ("bf16", 24), ("bf16", 7)])
+@pytest.mark.parametrize("dtype,C", [("f32", 5), ("f32", 32), ("f32", 44), ("bf16", 24), ("bf16", 7), ("bf16", 72)])
 def test_nchw_tensors(oracle, reduce, dtype, C):
     import torch
     w = wl.Workload(f"nchw{C}", 3000 + C, 2, 5, C, dtype, (10, 14), (80, 112), (17, 13, 6),
@@ -39,10 +39,17 @@ def test_nchw_tensors(oracle, reduce, dtype, C):
     f, m = _cuda_features(inp, fb.NCHW)
     X, Y, Z = w.grid
     cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=f.device)
-    out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, valid_count=cnt, layout=fb.NCHW)
-    assert fb.flashbev_last_kernel_name().startswith("per_output_nchw")
-    assert out.shape == (w.B, C, X, Y)
-    parity.assert_parity(w, ref, out.permute(0, 2, 3, 1).cpu().numpy(), cnt.cpu().numpy(), "[nchw]", check_fraction=False)
+    elem = 4 if dtype == "f32" else 2
+    for workspace in (True, False):
+        cnt.fill_(-1)
+        out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, valid_count=cnt, layout=fb.NCHW, workspace=workspace)
+        # with the scratch lent, shapes with whole 16-byte channel rows run the tiled kernel on a channels-last copy
+        tiled = workspace and (C * elem) % 16 == 0
+        assert fb.flashbev_last_kernel_name().startswith("tiled" if tiled else "per_output_nchw")
+        assert fb.flashbev_last_kernel_name().endswith("nchw" if tiled else ("bf16" if dtype == "bf16" else "f32"))
+        assert fb.flashbev_last_launch_count() == (2 if tiled else 1)
+        assert out.shape == (w.B, C, X, Y)
+        parity.assert_parity(w, ref, out.permute(0, 2, 3, 1).cpu().numpy(), cnt.cpu().numpy(), "[nchw]", check_fraction=False)
 
 
 def test_nchw_benchmark_shape(oracle):
@@ -52,7 +59,27 @@ def test_nchw_benchmark_shape(oracle):
     ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, EQ1)
     f, m = _cuda_features(inp, fb.NCHW)
     out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, EQ1, layout=fb.NCHW)
+    assert fb.flashbev_last_kernel_name() == "tiled_f32_nchw"
     parity.assert_parity(w, ref, out.permute(0, 2, 3, 1).cpu().numpy(), None, "[nchw tiny]")
+    # the planar result is the channels-last result, bit for bit (same kernel, same order of sums)
+    f2, _ = _cuda_features(inp, fb.NHWC)
+    out2 = fb.sampling_vt(f2, m, w.img_hw, w.bev_range, w.grid, EQ1)
+    assert torch.equal(out.permute(0, 2, 3, 1), out2)
+
+
+@pytest.mark.parametrize("name", ["representative", "half_taller"])
+def test_nchw_benchmark_configurations_on_the_tiled_kernel(oracle, name):
+    """Two benchmark configurations as channel-planar tensors (fp32 and bf16 features), against the oracle."""
+    import torch
+    w = wl.get(name)
+    inp = wl.make_inputs(w)
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, w.reduce)
+    f, m = _cuda_features(inp, fb.NCHW)
+    X, Y, Z = w.grid
+    cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=f.device)
+    out = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, w.reduce, valid_count=cnt, layout=fb.NCHW)
+    assert fb.flashbev_last_kernel_name().startswith("tiled") and fb.flashbev_last_kernel_name().endswith("nchw")
+    parity.assert_parity(w, ref, out.permute(0, 2, 3, 1).cpu().numpy(), cnt.cpu().numpy(), f"[nchw {name}]")
 
 
 @pytest.mark.parametrize("kernel", [fb.KERNEL_AUTO, fb.KERNEL_PER_OUTPUT])

@@ -531,6 +531,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 per-output, 2 tiled")
     ap.add_argument("--tune", type=str, default="0,0,0,0")
+    ap.add_argument("--backward-only", action="store_true",
+                    help="time flashbev_sampling_vt_backward on the workload's shape with fp32 gradients and print its own line "
+                         "(one GPU; what the backward profile under profiles/ was captured with)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = wl.get(args.workload)
@@ -563,6 +566,18 @@ def main():
     barrier()
     fb.lib()
     tune = tuple(int(t, 0) for t in args.tune.split(","))
+    if args.backward_only:
+        wb = wl.get(args.workload, dtype="f32")
+        lat = measure_backward(torch, wb, args, device, args.steps, args.warmup, barrier)
+        if rank == 0:
+            print(json.dumps({"metric": "sampling_vt_backward_latency", "value": lat, "unit": "ms", "higher_is_better": False,
+                              "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "dtype": "f32", "data": "synthetic",
+                              "config": {"workload": wb.name, "C": wb.C, "grid": list(wb.grid), "feat_hw": list(wb.feat_hw),
+                                         "launch": "cuda graph replay, memset + scatter kernel per frame"},
+                              "gpu_launches": args.steps * max(4, -(-3 * L2_BYTES // (wb.output_bytes + wb.B * wb.N * wb.feat_hw[0] * wb.feat_hw[1] * wb.C * 4)))}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # max over ranks of the device time of the K steps
     def reduce_max(x):

@@ -165,7 +165,9 @@ size_t flashbev_workspace_bytes(const flashbev_vt_params *p);
  */
 flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_staging,
                                           size_t staging_bytes, void *stream);
-size_t flashbev_host_staging_bytes(const flashbev_vt_params *p); /* 0 if `p` is invalid */
+/* 0 if `p` is invalid.  For NCHW tensors the figure includes flashbev_workspace_bytes(p) of scratch for the
+ * channels-last copy; a buffer without that last part is accepted and the generic kernel runs. */
+size_t flashbev_host_staging_bytes(const flashbev_vt_params *p);
 
 /*
  * Host-buffer variant that needs no device buffer from the caller and never allocates.
@@ -182,8 +184,9 @@ size_t flashbev_host_staging_bytes(const flashbev_vt_params *p); /* 0 if `p` is 
  * library image: every GPU on which the library is loaded sets that much memory aside until the
  * process exits, whether this function is used or not.
  *
- *  - A problem whose flashbev_host_staging_bytes(p) exceeds FLASHBEV_STATIC_STAGING_BYTES is
- *    refused with FLASHBEV_EXCEEDS_STATIC_STAGING before anything is enqueued.
+ *  - A problem whose flashbev_host_staging_bytes(p) (for NCHW tensors: without the optional scratch
+ *    part) exceeds FLASHBEV_STATIC_STAGING_BYTES is refused with FLASHBEV_EXCEEDS_STATIC_STAGING
+ *    before anything is enqueued.
  *  - The first call on each device looks up the device address of the array (once per device, with
  *    that device current) and remembers it; make that first call outside any stream capture.
  *  - The array is shared by every call and keeps whatever the previous call left in it.  Nothing in

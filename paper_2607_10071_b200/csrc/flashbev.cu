@@ -995,6 +995,7 @@ flashbev_status run_device(const flashbev_vt_params *p, cudaStream_t stream, boo
 
 struct StagingLayout {
     size_t feat_off, mat_off, out_off, cnt_off, total;
+    size_t ws_off, ws_bytes, total_with_ws;  // NCHW tensors: room for the channels-last copy behind the rest (optional)
 };
 
 // False if the staging area of this problem would not fit 2^62 bytes (the byte counts below would wrap).
@@ -1010,6 +1011,7 @@ bool staging_layout(const flashbev_vt_params *p, StagingLayout &s)
     s.out_off = s.mat_off + up((size_t)p->B * p->N * 64);
     s.cnt_off = s.out_off + up((size_t)p->B * p->X * p->Y * p->C * (p->out_dtype == FLASHBEV_F32 ? 4 : 2));
     s.total = s.cnt_off + (p->valid_count_out ? up((size_t)p->B * p->X * p->Y * 4) : 0);
+    s.ws_off = s.total, s.ws_bytes = nchw_copy_bytes(p), s.total_with_ws = s.total + up(s.ws_bytes);
     return true;
 }
 
@@ -1037,7 +1039,7 @@ size_t flashbev_host_staging_bytes(const flashbev_vt_params *p)
     flashbev_status st;
     if (!params_ok(p, st)) return 0;
     StagingLayout L;
-    return staging_layout(p, L) ? L.total : 0;
+    return staging_layout(p, L) ? L.total_with_ws : 0;
 }
 
 flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_staging, size_t staging_bytes,
@@ -1057,6 +1059,8 @@ flashbev_status flashbev_sampling_vt_host(const flashbev_vt_params *p, void *d_s
     d.lidar2img = reinterpret_cast<const float *>(base + L.mat_off);
     d.out = base + L.out_off;
     d.valid_count_out = p->valid_count_out ? reinterpret_cast<int32_t *>(base + L.cnt_off) : nullptr;
+    d.workspace = nullptr, d.workspace_bytes = 0;
+    if (L.ws_bytes && staging_bytes >= L.total_with_ws) d.workspace = base + L.ws_off, d.workspace_bytes = L.ws_bytes;
     const size_t feat_bytes =
         (size_t)p->B * p->N * p->feat_h * p->feat_w * p->C * (p->feat_dtype == FLASHBEV_F32 ? 4 : 2);
     if (cudaMemcpyAsync(base + L.feat_off, p->features, feat_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||

@@ -265,6 +265,33 @@ def test_host_buffer_entry_point(oracle, bench_inputs):
         parity.assert_parity(w, oracle_of(oracle, inp, w.reduce), hout.numpy(), hcnt.numpy(), "[host entry]")
 
 
+def test_host_buffer_entry_point_with_planar_tensors(oracle, bench_inputs):
+    """NCHW host tensors: with the whole staging area the channels-last copy is made there and the tiled kernel runs;
+    with the area cut down to its compulsory part the generic kernel runs; same numbers either way."""
+    import torch
+    inp = bench_inputs["tiny"]
+    w = inp.workload
+    X, Y, Z = w.grid
+    hf = torch.from_numpy(np.ascontiguousarray(inp.features.transpose(0, 1, 4, 2, 3))).pin_memory()
+    hm = torch.from_numpy(inp.lidar2img).pin_memory()
+    ref = oracle_of(oracle, inp, w.reduce)
+    full = None
+    for cut in (False, True):
+        hout = torch.full((w.B, w.C, X, Y), float("nan")).pin_memory()
+        p = fb.make_params(hf.data_ptr(), fb.F32, hm.data_ptr(), w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid,
+                           w.reduce, hout.data_ptr(), layout=fb.NCHW)
+        need, ws = fb.flashbev_host_staging_bytes(p), fb.flashbev_workspace_bytes(p)
+        assert ws == inp.features.nbytes and need >= w.unique_bytes + ws
+        staging = torch.empty(need, dtype=torch.uint8, device="cuda:0")
+        s = torch.cuda.Stream()
+        fb.flashbev_sampling_vt_host(p, staging.data_ptr(), need - ws if cut else need, s.cuda_stream)
+        s.synchronize()
+        assert fb.flashbev_last_kernel_name() == ("per_output_nchw_f32" if cut else "tiled_f32_nchw")
+        parity.assert_parity(w, ref, hout.permute(0, 2, 3, 1).numpy(), None, "[host entry, planar]")
+        full = hout if full is None else full
+    assert float((full - hout).abs().max()) <= 1e-5
+
+
 def test_runs_on_a_caller_stream(oracle, bench_inputs):
     import torch
     inp = bench_inputs["tiny"]

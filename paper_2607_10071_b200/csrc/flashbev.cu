@@ -257,26 +257,33 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
 
 // Kernel 1b: the same per-output decomposition for channel-planar tensors, features
 // [B][N][C][Hf][Wf] and out [B][C][X][Y] (the layout the paper's own kernel works on, Sec. 4.1:
-// C x Hf x Wf per camera, one thread per (b, x, y, c)).  Threads are ordered with iy fastest so
-// that stores and the taps of neighbouring cells coalesce.
-template <typename T>
+// C x Hf x Wf per camera).  One thread per (b, x, y, group of CH channels): the projection of a sample is shared by
+// the CH channel planes a thread reads.  Threads are ordered with iy fastest so that stores and the taps of
+// neighbouring cells coalesce.  Needs no scratch memory.
+template <typename T, int CH>
 __global__ void __launch_bounds__(256) vt_per_output_nchw_kernel(const KParams p)
 {
+    const int groups = (p.C + CH - 1) / CH;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (gid >= (long long)p.B * p.C * p.X * p.Y) return;
+    if (gid >= (long long)p.B * groups * p.X * p.Y) return;
     const int iy = (int)(gid % p.Y);
     const int ix = (int)((gid / p.Y) % p.X);
-    const int c = (int)((gid / ((long long)p.X * p.Y)) % p.C);
-    const int b = (int)(gid / ((long long)p.X * p.Y * p.C));
+    const int c0 = (int)((gid / ((long long)p.X * p.Y)) % groups) * CH;
+    const int b = (int)(gid / ((long long)p.X * p.Y * groups));
     const double xw = p.x_min + ((double)ix + 0.5) * p.dx;
     const double yw = p.y_min + ((double)iy + 0.5) * p.dy;
     const double wlim = (double)p.Wf - 0.5, hlim = (double)p.Hf - 0.5;
     const T *feat = static_cast<const T *>(p.feat);
-    float acc = 0.f;
+    const size_t plane_elems = (size_t)p.Hf * p.Wf;
+    float acc[CH];
+#pragma unroll
+    for (int j = 0; j < CH; ++j) acc[j] = 0.f;
     int count = 0;
     for (int k = 0; k < p.Z; ++k) {
         const double zw = p.z_min + ((double)k + 0.5) * p.dz;
-        float num = 0.f;
+        float num[CH];
+#pragma unroll
+        for (int j = 0; j < CH; ++j) num[j] = 0.f;
         int den = 0;
         for (int n = 0; n < p.N; ++n) {
             const float *M = p.l2i + ((size_t)b * p.N + n) * 16;
@@ -286,23 +293,39 @@ __global__ void __launch_bounds__(256) vt_per_output_nchw_kernel(const KParams p
             Sample s;
             if (!project_sample(p0 * p.sx, p1 * p.sy, d, wlim, hlim, s)) continue;
             den += 1;
-            const T *plane = feat + (((size_t)b * p.N + n) * p.C + c) * (size_t)p.Hf * p.Wf;
+            const T *plane = feat + (((size_t)b * p.N + n) * p.C + c0) * plane_elems;
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 const int xi = s.x0 + (t & 1), yi = s.y0 + (t >> 1);
                 if (xi < 0 || xi > p.Wf - 1 || yi < 0 || yi > p.Hf - 1) continue;  // zero padding
                 const float w = ((t & 1) ? s.tx : 1.f - s.tx) * ((t >> 1) ? s.ty : 1.f - s.ty);
-                num = fmaf(w, load_elem(plane + (size_t)yi * p.Wf + xi), num);
+                const T *tap = plane + (size_t)yi * p.Wf + xi;
+#pragma unroll
+                for (int j = 0; j < CH; ++j)
+                    if (c0 + j < p.C) num[j] = fmaf(w, load_elem(tap + j * plane_elems), num[j]);
             }
         }
         count += den;
-        if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) acc = fmaf(num, 1.f / (float)(den > 1 ? den : 1), acc);
-        else acc += num;
+        const float inv = 1.f / (float)(den > 1 ? den : 1);
+#pragma unroll
+        for (int j = 0; j < CH; ++j) {
+            if (p.reduce == FLASHBEV_REDUCE_CAMERA_MEAN_Z_SUM) acc[j] = fmaf(num[j], inv, acc[j]);
+            else acc[j] += num[j];
+        }
     }
-    if (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) acc *= 1.f / (float)(count > 1 ? count : 1);
-    if (p.out_bf16) reinterpret_cast<uint16_t *>(p.out)[gid] = __bfloat16_as_ushort(__float2bfloat16_rn(acc));
-    else p.out[gid] = p.accumulate ? acc + p.out[gid] : acc;
-    if (p.count_out && c == 0) p.count_out[((size_t)b * p.X + ix) * p.Y + iy] = count;
+    const float gn = p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID ? 1.f / (float)(count > 1 ? count : 1) : 1.f;
+    const size_t plane_out = (size_t)p.X * p.Y;
+    const size_t o0 = ((size_t)b * p.C + c0) * plane_out + (size_t)ix * p.Y + iy;
+#pragma unroll
+    for (int j = 0; j < CH; ++j) {
+        if (c0 + j >= p.C) break;
+        float v = acc[j];
+        if (p.reduce == FLASHBEV_REDUCE_MEAN_OVER_VALID) v *= gn;
+        const size_t o = o0 + j * plane_out;
+        if (p.out_bf16) reinterpret_cast<uint16_t *>(p.out)[o] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+        else p.out[o] = p.accumulate ? v + p.out[o] : v;
+    }
+    if (p.count_out && c0 == 0) p.count_out[((size_t)b * p.X + ix) * p.Y + iy] = count;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -674,11 +697,12 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
     const KParams k = base_params(p, accumulate);
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     if (p->layout == FLASHBEV_NCHW) {
-        const long long threads = (long long)p->B * p->C * p->X * p->Y;
+        constexpr int CH = 8;  // channel planes per thread
+        const long long threads = (long long)p->B * ((p->C + CH - 1) / CH) * p->X * p->Y;
         const long long blocks = (threads + 255) / 256;
         if (blocks > 2147483647LL) return FLASHBEV_UNSUPPORTED;
-        if (bf16) vt_per_output_nchw_kernel<uint16_t><<<dim3((unsigned)blocks), dim3(256), 0, stream>>>(k);
-        else vt_per_output_nchw_kernel<float><<<dim3((unsigned)blocks), dim3(256), 0, stream>>>(k);
+        if (bf16) vt_per_output_nchw_kernel<uint16_t, CH><<<dim3((unsigned)blocks), dim3(256), 0, stream>>>(k);
+        else vt_per_output_nchw_kernel<float, CH><<<dim3((unsigned)blocks), dim3(256), 0, stream>>>(k);
         t_last_kernel = bf16 ? "per_output_nchw_bf16" : "per_output_nchw_f32";
         return FLASHBEV_OK;
     }

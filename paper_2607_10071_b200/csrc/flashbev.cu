@@ -783,15 +783,15 @@ bool nchw_tiled_applicable(const flashbev_vt_params *p)
            (long long)p->B * p->N <= 65535 && (p->C + 31) / 32 <= 65535;
 }
 
-template <int V, bool BF16, int WARPS, bool BWD, bool WIDE = false>
+template <int V, bool BF16, int WARPS, bool BWD, bool WIDE = false, bool PLANAR = false>
 cudaError_t launch_tiled_inst(const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
 {
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE>,
+        cudaError_t e = cudaFuncSetAttribute(vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE, PLANAR>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
+    vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE, PLANAR><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
     return cudaSuccess;
 }
 
@@ -803,6 +803,10 @@ cudaError_t launch_tiled_warps(int warps, const KParams &k, dim3 grid, size_t sm
         case 2: return launch_tiled_inst<V, BF16, 2, false>(k, grid, smem, stream);
         case 8: return launch_tiled_inst<V, BF16, 8, false>(k, grid, smem, stream);
         default:
+            if (k.out_nchw) {  // (planar output: instances for 4 warps per CTA only)
+                if (V >= 2 && k.wide) return launch_tiled_inst<V, BF16, 4, false, (V >= 2), true>(k, grid, smem, stream);
+                return launch_tiled_inst<V, BF16, 4, false, false, true>(k, grid, smem, stream);
+            }
             if (V >= 2 && k.wide) return launch_tiled_inst<V, BF16, 4, false, (V >= 2)>(k, grid, smem, stream);
             return launch_tiled_inst<V, BF16, 4, false>(k, grid, smem, stream);
     }
@@ -964,6 +968,7 @@ flashbev_status launch_nchw_tiled(const flashbev_vt_params *p, cudaStream_t stre
     flashbev_vt_params q = *p;
     q.features = p->workspace;
     q.layout = FLASHBEV_NHWC;
+    q.tune[3] = (q.tune[3] & ~0xf) | 4;  // the planar-output instances are built for 4 warps per CTA
     {   // configure first: nothing is enqueued for a shape the tiled kernel cannot take
         KParams k;
         int V, warps;

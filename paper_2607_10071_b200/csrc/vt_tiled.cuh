@@ -698,7 +698,9 @@ __device__ __forceinline__ void walk_one(const KParams &p, const WarpSmem &sm, c
 }
 
 // WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
-template <int V, bool BF16, int WARPS, bool BWD, bool WIDE>
+// PLANAR: the output is [B][C][X][Y] (the features are a channels-last copy of planar ones); instances of their own, so
+// that the channels-last instances do not carry the scalar stores
+template <int V, bool BF16, int WARPS, bool BWD, bool WIDE, bool PLANAR = false>
 __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / WARPS)
     vt_tiled_kernel(const KParams p)
 {
@@ -919,7 +921,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                             for (int e = 0; e < PV; ++e) acc[v][e].x *= gn, acc[v][e].y *= gn;
                     }
                     float *o = p.out + ocell * p.C + out_lane;  // this lane's first channel of the cell
-                    if (p.out_nchw) {
+                    if (PLANAR) {
                         // channel-planar output [B][C][X][Y]: one scalar per channel, the cells of a sub-block adjacent in y
                         const size_t plane = (size_t)p.X * p.Y;
                         const size_t at = ocell + (size_t)b * plane * (size_t)(p.C - 1);  // b C plane + (cell inside the batch element)

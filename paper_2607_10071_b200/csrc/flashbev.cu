@@ -153,8 +153,10 @@ __device__ __forceinline__ float load_elem(const uint16_t *p)
 
 // ------------------------------------------------------------------------------------------
 // Kernel 1: one thread per (cell, group of VEC channels).  T = float or uint16_t (bf16 bits).
+// SCALAR: the group's channels are loaded and stored one by one (any channel count, any alignment; the last group may
+// be short); otherwise as one 16-byte vector.
 
-template <typename T, int VEC>
+template <typename T, int VEC, bool SCALAR = false>
 __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
 {
     const int groups = (p.C + VEC - 1) / VEC;
@@ -196,8 +198,10 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
                 if (xi < 0 || xi > p.Wf - 1 || yi < 0 || yi > p.Hf - 1) continue;  // zero padding
                 const float w = ((t & 1) ? s.tx : 1.f - s.tx) * ((t >> 1) ? s.ty : 1.f - s.ty);
                 const T *tp = fn + ((size_t)yi * p.Wf + xi) * p.C + c0;
-                if (VEC == 1) {
-                    num[0] = fmaf(w, load_elem(tp), num[0]);
+                if (SCALAR) {
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i)
+                        if (c0 + i < p.C) num[i] = fmaf(w, load_elem(tp + i), num[i]);
                 } else if (sizeof(T) == 4) {
                     const float4 v = __ldg(reinterpret_cast<const float4 *>(tp));
                     num[0] = fmaf(w, v.x, num[0]);
@@ -229,8 +233,10 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
     }
     if (p.out_bf16) {
         uint16_t *o = reinterpret_cast<uint16_t *>(p.out) + (size_t)cell * p.C + c0;
-        if (VEC == 1) {
-            o[0] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[0]));
+        if (SCALAR) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i)
+                if (c0 + i < p.C) o[i] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[i]));
         } else {
 #pragma unroll
             for (int i = 0; i < VEC; i += 4)
@@ -241,10 +247,13 @@ __global__ void __launch_bounds__(256) vt_per_output_kernel(const KParams p)
         float *o = p.out + (size_t)cell * p.C + c0;
         if (p.accumulate) {
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) acc[i] += o[i];
+            for (int i = 0; i < VEC; ++i)
+                if (!SCALAR || c0 + i < p.C) acc[i] += o[i];
         }
-        if (VEC == 1) {
-            o[0] = acc[0];
+        if (SCALAR) {
+#pragma unroll
+            for (int i = 0; i < VEC; ++i)
+                if (c0 + i < p.C) o[i] = acc[i];
         } else {
 #pragma unroll
             for (int i = 0; i < VEC; i += 4)
@@ -708,7 +717,8 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
     }
     const int vec = bf16 ? 8 : 4;
     const bool vec_ok = (p->C % vec == 0) && ((uintptr_t)p->features % 16 == 0) && ((uintptr_t)p->out % 16 == 0);
-    const int per_thread = vec_ok ? vec : 1;
+    constexpr int kScalarGroup = 4;  // channels per thread when they are loaded one by one
+    const int per_thread = vec_ok ? vec : kScalarGroup;
     const long long threads = (long long)p->B * p->X * p->Y * ((p->C + per_thread - 1) / per_thread);
     const long long blocks = (threads + 255) / 256;
     if (blocks > 2147483647LL) return FLASHBEV_UNSUPPORTED;
@@ -717,13 +727,13 @@ flashbev_status launch_per_output(const flashbev_vt_params *p, cudaStream_t stre
         vt_per_output_kernel<uint16_t, 8><<<grid, block, 0, stream>>>(k);
         t_last_kernel = "per_output_bf16x8";
     } else if (bf16) {
-        vt_per_output_kernel<uint16_t, 1><<<grid, block, 0, stream>>>(k);
+        vt_per_output_kernel<uint16_t, kScalarGroup, true><<<grid, block, 0, stream>>>(k);
         t_last_kernel = "per_output_bf16x1";
     } else if (vec_ok) {
         vt_per_output_kernel<float, 4><<<grid, block, 0, stream>>>(k);
         t_last_kernel = "per_output_f32x4";
     } else {
-        vt_per_output_kernel<float, 1><<<grid, block, 0, stream>>>(k);
+        vt_per_output_kernel<float, kScalarGroup, true><<<grid, block, 0, stream>>>(k);
         t_last_kernel = "per_output_f32x1";
     }
     return FLASHBEV_OK;

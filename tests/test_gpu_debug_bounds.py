@@ -8,6 +8,7 @@ require the word to stay 0 and the results to match the oracle as in the normal 
 """
 import numpy as np
 import pytest
+from hypothesis import HealthCheck, given, settings, strategies as st
 
 from paper_2607_10071_b200 import binding as fb
 from paper_2607_10071_b200 import build as fbuild
@@ -116,3 +117,42 @@ def test_backward_makes_no_out_of_range_index(checked, name, C, reduce, tune3):
     assert int(word.item()) == 0
     scale = float(ref.abs().max())
     assert float((gf - ref).abs().max()) <= 1e-5 * max(1.0, scale)
+
+
+@st.composite
+def checked_cases(draw):
+    dtype = draw(st.sampled_from(["f32", "bf16"]))
+    vec = 4 if dtype == "f32" else 8
+    return dict(
+        seed=draw(st.integers(0, 10_000)), dtype=dtype, C=vec * draw(st.sampled_from([1, 2, 3, 5, 8, 10, 16, 20, 33])),
+        B=draw(st.integers(1, 2)), N=draw(st.integers(1, 9)),
+        feat=(draw(st.integers(1, 20)), draw(st.integers(1, 24))),
+        grid=(draw(st.integers(1, 19)), draw(st.integers(1, 19)), draw(st.sampled_from([1, 2, 5, 8, 16, 40, 97, 200]))),
+        general=draw(st.booleans()), rng_xy=draw(st.sampled_from([3.0, 10.0, 40.0])),
+        reduce=draw(st.sampled_from([0, 1, 2])),
+        walk=draw(st.sampled_from([0, 1, 4, 16, 64])), slots=draw(st.sampled_from([0, 64, 96, 256, 1024])),
+        shape=draw(st.sampled_from([0, (1 << 4) | (1 << 8), (2 << 4) | (2 << 8), (4 << 4) | (4 << 8)])),
+        tail=draw(st.integers(0, 7)), order=draw(st.sampled_from([0, 1 << 28, 1 << 18, 3 << 18])))
+
+
+@settings(max_examples=50, deadline=None, derandomize=True,
+          suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
+@given(case=checked_cases())
+def test_random_problems_and_hints_make_no_out_of_range_index(oracle, checked, case):
+    """Random rigs (surround and general pose), shapes, dtypes, reduce modes and launch-geometry hints -- small record
+    lists that force many rounds, long and short runs, every order of the work -- in the bounds-checked build: no index
+    out of range, and the oracle's numbers."""
+    w = wl.Workload("checked", 9000 + case["seed"], case["B"], case["N"], case["C"], case["dtype"], case["feat"],
+                    (case["feat"][0] * 8, case["feat"][1] * 8), case["grid"],
+                    (-case["rng_xy"], case["rng_xy"], -case["rng_xy"], case["rng_xy"], -3.0, 2.5), case["reduce"],
+                    general_pose=case["general"], yaw_jitter_deg=5.0)
+    inp = wl.make_inputs(w)
+    tune = (0, 0, case["walk"], case["shape"] | ((case["slots"] // 16) << 20) | (case["tail"] << 29) | case["order"])
+    try:
+        out, cnt, violations = run_checked(checked, inp, case["reduce"], tune)
+    except fb.FlashBevError as e:  # hints the forced tiled kernel cannot be configured for: refused on the host
+        assert e.status == fb.UNSUPPORTED, e
+        return
+    assert violations == 0, f"{case}: {violations} out-of-range indices"
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, case["reduce"])
+    parity.assert_parity(w, ref, out, cnt, f"[checked build {case}]", check_fraction=False, large_outputs=True)

@@ -146,6 +146,10 @@ typedef struct flashbev_vt_params {
  * (two for NCHW tensors with a workspace: a transposing copy first) and returns without waiting
  * (`stream` is a cudaStream_t, passed as void*; NULL = the default stream).
  * Uses no device memory beyond `features`, `lidar2img`, `out`, `valid_count_out` and `workspace`.
+ * The tiled kernel is launched with programmatic stream serialization: its thread blocks may be
+ * placed on the SMs while the kernel before it in the stream is still draining, and wait there for
+ * that kernel's completion before they read or write any global memory -- stream order as seen
+ * through memory is unchanged.  The environment variable FLASHBEV_NO_PDL turns this off.
  */
 flashbev_status flashbev_sampling_vt(const flashbev_vt_params *p, void *stream);
 

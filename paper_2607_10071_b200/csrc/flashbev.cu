@@ -45,6 +45,7 @@ struct KParams {
     int B, N, C, Hf, Wf, X, Y, Z, reduce;
     int out_bf16;               // store the output as bfloat16 (round to nearest even) instead of float32
     int out_nchw;               // tiled kernel: the output is [B][C][X][Y] (scalar stores), features are a channels-last copy
+    int pdl;                    // host only: launch the forward with programmatic stream serialization
     int accumulate;             // add the result to the fp32 output instead of overwriting it (multi-resolution levels)
     double sx, sy;              // image px -> feature px
     double x_min, dx, y_min, dy, z_min, dz;
@@ -801,6 +802,17 @@ cudaError_t launch_tiled_inst(const KParams &k, dim3 grid, size_t smem, cudaStre
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
+    if (!BWD && k.pdl) {
+        // forward launches may overlap their start with the end of the kernel before them in the stream (the kernel
+        // waits for that kernel's completion before it reads or writes global memory)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid, cfg.blockDim = dim3(WARPS * 32), cfg.dynamicSmemBytes = smem, cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr, cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE, PLANAR>, k);
+    }
     vt_tiled_kernel<V, BF16, WARPS, BWD, WIDE, PLANAR><<<grid, dim3(WARPS * 32), smem, stream>>>(k);
     return cudaSuccess;
 }
@@ -955,6 +967,7 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, b
     const flashbev_status st = configure_tiled(p, k, V, warps, grid, smem, accumulate);
     if (st != FLASHBEV_OK) return st;
     k.out_nchw = out_nchw;
+    k.pdl = getenv("FLASHBEV_NO_PDL") ? 0 : 1;
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     cudaError_t e;
     static const char *const names[2][3] = {{"tiled_f32_v1", "tiled_f32_v2", "tiled_f32_v4"},

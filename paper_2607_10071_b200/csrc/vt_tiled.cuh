@@ -721,6 +721,14 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                    warp * warp_smem_layout(nullptr, nullptr, p.slots, p.colcap, p.wcap, p.ct, p.ct * p.N, p.den_bytes);
     const WarpSmem sm = warp_smem(p, cx.warp_base);
 
+    // Programmatic dependent launch: let the next grid of the stream place its CTAs while this one drains, and (as the
+    // dependent of the grid before) touch no global memory until that grid has completed and its writes are visible.
+    // Both are no-ops for a launch without the attribute.
+    if (!BWD) {
+        asm volatile("griddepcontrol.launch_dependents;");
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+
     // ---- per-CTA tables: camera matrices (scaled to feature texels), condition slopes, camera class, cell positions
     for (int i = tid; i < p.N * 12; i += THREADS) {
         const int n = i / 12, e = i - n * 12;

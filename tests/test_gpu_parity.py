@@ -306,3 +306,38 @@ def test_runs_on_a_caller_stream(oracle, bench_inputs):
     s.synchronize()
     assert fb.flashbev_last_launch_count() == 1
     parity.assert_parity(w, oracle_of(oracle, inp, SUM), out.cpu().numpy(), None)
+
+
+def test_back_to_back_launches_keep_stream_order(bench_inputs):
+    """The forward is launched with programmatic stream serialization (its thread blocks may be resident before the
+    kernel in front of it has finished).  A second call that reads the first call's output as its feature map must see
+    the finished output: same bits as with a synchronisation in between, over many rounds with changing inputs."""
+    import torch
+    inp = bench_inputs["tiny"]
+    w = inp.workload
+    dev = torch.device("cuda:0")
+    X, Y, Z = w.grid
+    mats = torch.from_numpy(inp.lidar2img).to(dev)
+    w2 = wl.Workload("chained", 4242, 1, 1, w.C, "f32", (X, Y), (X * 8, Y * 8), (64, 64, 8),
+                     (-20.0, 20.0, -20.0, 20.0, -3.0, 3.0), 0, general_pose=False, yaw_jitter_deg=0.0, fov_deg=100.0)
+    mats2 = torch.from_numpy(wl.make_inputs(w2).lidar2img).to(dev)
+    g = torch.Generator(device=dev).manual_seed(5)
+    stream = torch.cuda.Stream(dev)
+    for it in range(20):
+        feats = torch.randn((w.B, w.N) + tuple(w.feat_hw) + (w.C,), generator=g, device=dev)
+        mid = torch.zeros((1, X, Y, w.C), device=dev)
+        outs = []
+        for synced in (True, False):
+            mid.zero_()
+            out2 = torch.full((1, 64, 64, w.C), float("nan"), device=dev)
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream):
+                fb.sampling_vt(feats, mats, w.img_hw, w.bev_range, w.grid, 0, out=mid, stream=stream.cuda_stream)
+                if synced:
+                    stream.synchronize()
+                fb.sampling_vt(mid.view(1, 1, X, Y, w.C), mats2, w2.img_hw, w2.bev_range, w2.grid, 0, out=out2,
+                               stream=stream.cuda_stream)
+            stream.synchronize()
+            outs.append(out2)
+        assert torch.equal(outs[0], outs[1]), it
+        assert float(outs[0].abs().max()) > 0.0

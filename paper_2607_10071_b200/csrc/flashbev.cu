@@ -853,9 +853,7 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     if (!(V == 1 || V == 2 || V == 4) || g < 1 || g > 32) V = 0, g = 0;
     if (!V) {
         // (measured) up to 8 vectors per texel: one per lane; up to 32: two adjacent ones per lane; beyond: four.
-        // Tall columns of 8-vector texels: eight cells per sub-block amortise the geometry better.
-        if (k.vecs == 8 && p->Z >= 32 && (long long)p->B * p->X * p->Y >= 65536) V = 2, g = 4;
-        else if (k.vecs <= 8) V = 1, g = k.vecs;
+        if (k.vecs <= 8) V = 1, g = k.vecs;
         else if (k.vecs <= 32) V = (k.vecs % 2 == 0 || k.vecs > 16) ? 2 : 1, g = (k.vecs + V - 1) / V;
         else V = 4, g = (k.vecs + 3) / 4;
         if (g > 32) g = 32;
@@ -902,13 +900,16 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     };
     if (sbx < 1 || sby < 1 || !fits(sbx, sby)) {
         // (from sweeps) about 10-16 cells per warp -- enough columns to keep the geometry lanes busy -- but fewer if
-        // that leaves the SMs less than three rounds of warps, never more than the record slots hold in one round
-        // (a cell writes roughly 1.2 Z + 12 records on surround rigs) and never fewer warps than the SMs can hold.
+        // that leaves the SMs less than three rounds of warps, never more than the record slots hold in four rounds
+        // (a cell writes roughly 1.2 Z + 12 records on surround rigs; rounds hold whole sub-blocks, and columns of
+        // 32-256 bins gain more from full geometry lanes than they lose to further rounds: 20-30 % measured) and
+        // never fewer warps than the SMs can hold.
         static const int shapes[][2] = {{1, 1}, {1, 2}, {2, 2}, {2, 3}, {2, 4}, {3, 3}, {3, 4}, {4, 4}};
         const long long cells = (long long)p->B * p->X * p->Y, warp_slots = (long long)sm_count() * 20;
         double want = std::min(16.0, std::max(10.0, (double)cells / (3.0 * warp_slots)));
         want = std::min(want, (double)cells / warp_slots);
-        want = std::min(want, k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0));
+        const double rounds = p->Z <= 5 * p->feat_h ? 4.0 : 1.0;  // (very tall columns: the walkers dominate, one round is better)
+        want = std::min(want, rounds * k.slots / (1.2 * std::min(p->Z, 2 * p->feat_h) + 12.0));
         sbx = sby = 1;
         double best = 1e30;
         for (const auto &sh : shapes) {

@@ -131,12 +131,14 @@ typedef struct flashbev_vt_params {
                                   dereferenced.  The caller zeroes the word before the call and reads it after
                                   synchronising.  The normal build ignores it.  Callers built against an older
                                   header (struct_size without this field) are accepted. */
-    void *workspace;           /* optional DEVICE scratch, 16-byte aligned, or NULL.  Only channel-planar (NCHW)
-                                  tensors use it: with flashbev_workspace_bytes(p) bytes here the features are
-                                  first transposed into it (channels last) and the tiled kernel runs on the copy,
-                                  writing the NCHW output directly; without it NCHW tensors take the generic
-                                  per-output kernel (an order of magnitude slower).  Callers built against a
-                                  header without these two fields are accepted. */
+    void *workspace;           /* optional DEVICE scratch, 16-byte aligned, or NULL.  Two kinds of tensors use it,
+                                  with flashbev_workspace_bytes(p) bytes here: channel-planar (NCHW) features are
+                                  first transposed into it (channels last), and channels-last features whose rows
+                                  are not whole 16-byte vectors are copied into it with zero-padded rows; the
+                                  tiled kernel then runs on the copy and writes the output in the caller's own
+                                  layout.  Without it such tensors take the generic per-output kernel (several
+                                  times to an order of magnitude slower).  Callers built against a header without
+                                  these two fields are accepted. */
     size_t workspace_bytes;    /* size of `workspace` */
 } flashbev_vt_params;
 
@@ -154,9 +156,10 @@ typedef struct flashbev_vt_params {
 flashbev_status flashbev_sampling_vt(const flashbev_vt_params *p, void *stream);
 
 /* Device scratch the operator can use beyond its inputs and outputs.  0 for channels-last (NHWC)
- * tensors (Sec. 3.3.1: all intermediates live in registers / on chip).  For NCHW tensors whose
- * channel rows are whole 16-byte vectors: the size of a channels-last copy of the features, which
- * `workspace` may lend to the call (optional; see the field). */
+ * tensors with rows of whole 16-byte vectors (Sec. 3.3.1: all intermediates live in registers / on
+ * chip).  For NCHW tensors with such rows: the size of a channels-last copy of the features; for
+ * channels-last tensors with other channel counts: the size of a copy with the rows padded to whole
+ * vectors.  `workspace` may lend it to the call (optional; see the field). */
 size_t flashbev_workspace_bytes(const flashbev_vt_params *p);
 
 /*

@@ -354,8 +354,9 @@ def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM,
     """features: CUDA tensor [B,N,Hf,Wf,C] (NHWC) or [B,N,C,Hf,Wf] (NCHW), float32 or bfloat16,
     contiguous; lidar2img: CUDA float32 [B,N,4,4].  Returns the output tensor [B,X,Y,C] (NHWC) or
     [B,C,X,Y] (NCHW), float32 or bfloat16 per ``out_dtype`` (allocated by torch if ``out`` is None).
-    ``workspace``: for NCHW tensors, lend the call the scratch ``flashbev_workspace_bytes`` asks for (a torch
-    allocation, or a uint8 CUDA tensor of the caller's); False: none, the generic kernel runs."""
+    ``workspace``: for NCHW tensors and for channel counts that are not whole 16-byte vectors, lend the call the
+    scratch ``flashbev_workspace_bytes`` asks for (a torch allocation, or a uint8 CUDA tensor of the caller's);
+    False: none, the generic kernel runs."""
     import torch
 
     if not features.is_cuda or not lidar2img.is_cuda:
@@ -381,7 +382,7 @@ def sampling_vt(features, lidar2img, img_hw, bev_range, grid, reduce=REDUCE_SUM,
     p = make_params(features.data_ptr(), dt, lidar2img.data_ptr(), B, N, C, (Hf, Wf), img_hw, bev_range,
                     (X, Y, Z), reduce, out.data_ptr(),
                     None if valid_count is None else valid_count.data_ptr(), kernel, tune, layout, out_dtype)
-    if layout == NCHW and workspace is not False and workspace is not None:
+    if workspace is not False and workspace is not None:
         need = flashbev_workspace_bytes(p)
         if need:
             ws = workspace if workspace is not True else torch.empty(need, dtype=torch.uint8, device=features.device)

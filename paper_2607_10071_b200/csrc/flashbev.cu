@@ -44,7 +44,9 @@ struct KParams {
     float *gfeat;               // backward: gradient of the features [B][N][Hf][Wf][C], fp32, pre-zeroed
     int B, N, C, Hf, Wf, X, Y, Z, reduce;
     int out_bf16;               // store the output as bfloat16 (round to nearest even) instead of float32
-    int out_nchw;               // tiled kernel: the output is [B][C][X][Y] (scalar stores), features are a channels-last copy
+    int out_nchw;               // tiled kernel: scalar stores with the strides below (planar output, or ragged channels-last rows)
+    int out_c;                  // ... channels of the output (the kernel's C may be padded)
+    size_t out_bs, out_cells, out_chs;  // ... element strides of batch element, cell and channel
     int pdl;                    // host only: launch the forward with programmatic stream serialization
     int accumulate;             // add the result to the fp32 output instead of overwriting it (multi-resolution levels)
     double sx, sy;              // image px -> feature px
@@ -623,6 +625,18 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const T *__restrict__
     }
 }
 
+// Channels-last rows of C elements -> rows of Cpad >= C elements, the tail zero (T: 2- or 4-byte elements).
+template <typename T>
+__global__ void __launch_bounds__(256) pad_channels_kernel(const T *__restrict__ in, T *__restrict__ out, long long rows, int C, int Cpad)
+{
+    const long long total = rows * Cpad;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / Cpad;
+        const int c = (int)(i - r * Cpad);
+        out[i] = c < C ? in[r * C + c] : T(0);
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // host side
 
@@ -794,6 +808,31 @@ bool nchw_tiled_applicable(const flashbev_vt_params *p)
            (long long)p->B * p->N <= 65535 && (p->C + 31) / 32 <= 65535;
 }
 
+// Channels-last tensors whose rows are not whole 16-byte vectors: channels rounded up to the next whole vector.
+int padded_channels(const flashbev_vt_params *p)
+{
+    const int vec = p->feat_dtype == FLASHBEV_F32 ? 4 : 8;
+    return (p->C + vec - 1) / vec * vec;
+}
+
+// Bytes of the padded copy of such features (0: not that case, or the padded shape cannot take the tiled kernel).
+size_t pad_copy_bytes(const flashbev_vt_params *p)
+{
+    const size_t elem = p->feat_dtype == FLASHBEV_F32 ? 4 : 2;
+    if (p->layout != FLASHBEV_NHWC || ((size_t)p->C * elem) % 16 == 0) return 0;
+    flashbev_vt_params q = copy_params(p);
+    q.C = padded_channels(p);
+    if (!tiled_shape_ok(&q)) return 0;
+    return (size_t)p->B * p->N * p->feat_h * p->feat_w * q.C * elem;
+}
+
+bool padded_tiled_applicable(const flashbev_vt_params *p)
+{
+    if (p->struct_size < sizeof(flashbev_vt_params) || !p->workspace) return false;
+    const size_t need = pad_copy_bytes(p);
+    return need && p->workspace_bytes >= need && (uintptr_t)p->workspace % 16 == 0;
+}
+
 template <int V, bool BF16, int WARPS, bool BWD, bool WIDE = false, bool PLANAR = false>
 cudaError_t launch_tiled_inst(const KParams &k, dim3 grid, size_t smem, cudaStream_t stream)
 {
@@ -959,7 +998,10 @@ flashbev_status configure_tiled(const flashbev_vt_params *p, KParams &k, int &V,
     return FLASHBEV_OK;
 }
 
-flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false, bool out_nchw = false)
+// scalar_out: 0 vector stores into channels-last rows; 1 planar output [B][C][X][Y]; 2 channels-last rows of out_c
+// channels (the kernel's own C is padded)
+flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false, int scalar_out = 0,
+                             int out_c = 0)
 {
     KParams k;
     int V, warps;
@@ -967,7 +1009,12 @@ flashbev_status launch_tiled(const flashbev_vt_params *p, cudaStream_t stream, b
     size_t smem;
     const flashbev_status st = configure_tiled(p, k, V, warps, grid, smem, accumulate);
     if (st != FLASHBEV_OK) return st;
-    k.out_nchw = out_nchw;
+    k.out_nchw = scalar_out != 0;
+    {
+        const size_t plane = (size_t)p->X * p->Y;
+        if (scalar_out == 1) k.out_c = p->C, k.out_bs = plane * p->C, k.out_cells = 1, k.out_chs = plane;
+        if (scalar_out == 2) k.out_c = out_c, k.out_bs = plane * out_c, k.out_cells = out_c, k.out_chs = 1;
+    }
     k.pdl = getenv("FLASHBEV_NO_PDL") ? 0 : 1;
     const bool bf16 = p->feat_dtype == FLASHBEV_BF16;
     cudaError_t e;
@@ -1010,14 +1057,53 @@ flashbev_status launch_nchw_tiled(const flashbev_vt_params *p, cudaStream_t stre
         nchw_to_nhwc_kernel<float><<<grid, block, 0, stream>>>(static_cast<const float *>(p->features),
                                                                static_cast<float *>(p->workspace), p->C, HW);
     if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
-    const flashbev_status st = launch_tiled(&q, stream, accumulate, true);
+    const flashbev_status st = launch_tiled(&q, stream, accumulate, 1);
     if (st == FLASHBEV_OK) t_last_kernel = p->feat_dtype == FLASHBEV_BF16 ? "tiled_bf16_nchw" : "tiled_f32_nchw";
+    return st;
+}
+
+// Ragged channels-last tensors on the tiled kernel: features -> zero-padded copy in the workspace, output written
+// one channel at a time into the caller's rows.
+flashbev_status launch_padded_tiled(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate)
+{
+    flashbev_vt_params q = *p;
+    q.features = p->workspace;
+    q.C = padded_channels(p);
+    q.tune[3] = (q.tune[3] & ~0xf) | 4;  // the scalar-store instances are built for 4 warps per CTA
+    {
+        KParams k;
+        int V, warps;
+        dim3 grid;
+        size_t smem;
+        const flashbev_status st = configure_tiled(&q, k, V, warps, grid, smem, accumulate);
+        if (st != FLASHBEV_OK) return st;
+    }
+    const long long rows = (long long)p->B * p->N * p->feat_h * p->feat_w;
+    const unsigned blocks = (unsigned)std::min<long long>((rows * q.C + 255) / 256, 148LL * 32);
+    if (p->feat_dtype == FLASHBEV_BF16)
+        pad_channels_kernel<uint16_t><<<blocks, 256, 0, stream>>>(static_cast<const uint16_t *>(p->features),
+                                                                  static_cast<uint16_t *>(p->workspace), rows, p->C, q.C);
+    else
+        pad_channels_kernel<float><<<blocks, 256, 0, stream>>>(static_cast<const float *>(p->features),
+                                                               static_cast<float *>(p->workspace), rows, p->C, q.C);
+    if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+    const flashbev_status st = launch_tiled(&q, stream, accumulate, 2, p->C);
+    if (st == FLASHBEV_OK) t_last_kernel = p->feat_dtype == FLASHBEV_BF16 ? "tiled_bf16_padded" : "tiled_f32_padded";
     return st;
 }
 
 flashbev_status run_device(const flashbev_vt_params *p, cudaStream_t stream, bool accumulate = false)
 {
     flashbev_status st;
+    if (p->layout == FLASHBEV_NHWC && p->kernel != FLASHBEV_KERNEL_PER_OUTPUT && padded_tiled_applicable(p)) {
+        st = launch_padded_tiled(p, stream, accumulate);
+        if (st == FLASHBEV_OK) {
+            if (cudaGetLastError() != cudaSuccess) return FLASHBEV_CUDA_ERROR;
+            t_last_launches = 2;
+            return FLASHBEV_OK;
+        }
+        if (!(st == FLASHBEV_UNSUPPORTED && p->kernel == FLASHBEV_KERNEL_AUTO)) return st;
+    }
     if (p->layout == FLASHBEV_NCHW) {
         const bool can = nchw_tiled_applicable(p);
         if (p->kernel == FLASHBEV_KERNEL_TILED && !can) return FLASHBEV_UNSUPPORTED;
@@ -1064,7 +1150,8 @@ bool staging_layout(const flashbev_vt_params *p, StagingLayout &s)
     s.out_off = s.mat_off + up((size_t)p->B * p->N * 64);
     s.cnt_off = s.out_off + up((size_t)p->B * p->X * p->Y * p->C * (p->out_dtype == FLASHBEV_F32 ? 4 : 2));
     s.total = s.cnt_off + (p->valid_count_out ? up((size_t)p->B * p->X * p->Y * 4) : 0);
-    s.ws_off = s.total, s.ws_bytes = nchw_copy_bytes(p), s.total_with_ws = s.total + up(s.ws_bytes);
+    s.ws_off = s.total, s.ws_bytes = p->layout == FLASHBEV_NCHW ? nchw_copy_bytes(p) : pad_copy_bytes(p);
+    s.total_with_ws = s.total + up(s.ws_bytes);
     return true;
 }
 
@@ -1084,7 +1171,7 @@ size_t flashbev_workspace_bytes(const flashbev_vt_params *p)
 {
     flashbev_status st;
     if (!params_ok(p, st)) return 0;
-    return nchw_copy_bytes(p);
+    return p->layout == FLASHBEV_NCHW ? nchw_copy_bytes(p) : pad_copy_bytes(p);
 }
 
 size_t flashbev_host_staging_bytes(const flashbev_vt_params *p)

@@ -698,8 +698,9 @@ __device__ __forceinline__ void walk_one(const KParams &p, const WarpSmem &sm, c
 }
 
 // WIDE: a lane's V channel vectors are adjacent (32-byte aligned pairs, 256-bit loads) instead of g apart
-// PLANAR: the output is [B][C][X][Y] (the features are a channels-last copy of planar ones); instances of their own, so
-// that the channels-last instances do not carry the scalar stores
+// PLANAR: the output is written one channel at a time with the strides in the parameters -- [B][C][X][Y] tensors, or
+// channels-last rows that are not whole 16-byte vectors (the features are then a copy in the kernel's own layout);
+// instances of their own, so that the vector-store instances do not carry the scalar stores
 template <int V, bool BF16, int WARPS, bool BWD, bool WIDE, bool PLANAR = false>
 __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / WARPS)
     vt_tiled_kernel(const KParams p)
@@ -930,9 +931,10 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                     }
                     float *o = p.out + ocell * p.C + out_lane;  // this lane's first channel of the cell
                     if (PLANAR) {
-                        // channel-planar output [B][C][X][Y]: one scalar per channel, the cells of a sub-block adjacent in y
+                        // one scalar per channel: out[b][cell][channel] with the strides of the caller's layout (planar:
+                        // the cells of a sub-block are adjacent in y; ragged channels-last rows: channels adjacent)
                         const size_t plane = (size_t)p.X * p.Y;
-                        const size_t at = ocell + (size_t)b * plane * (size_t)(p.C - 1);  // b C plane + (cell inside the batch element)
+                        const size_t at = (size_t)b * p.out_bs + (ocell - (size_t)b * plane) * p.out_cells;
 #pragma unroll
                         for (int v = 0; v < V; ++v)
                             if (von[v]) {
@@ -940,7 +942,9 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                                 for (int e = 0; e < PV; ++e) {
 #pragma unroll
                                     for (int hl = 0; hl < 2; ++hl) {
-                                        const size_t idx = at + (size_t)(out_lane + v * vstride + e * 2 + hl) * plane;
+                                        const int ch = out_lane + v * vstride + e * 2 + hl;
+                                        if (ch >= p.out_c) continue;  // (padding channels of the copy)
+                                        const size_t idx = at + (size_t)ch * p.out_chs;
                                         float val = hl ? acc[v][e].y : acc[v][e].x;
                                         if (p.out_bf16) {
                                             uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + idx;

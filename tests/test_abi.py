@@ -122,6 +122,9 @@ def test_workspace_is_asked_for_planar_tensors_only():
     assert fb.flashbev_workspace_bytes(good_params()) == 0
     assert fb.flashbev_workspace_bytes(good_params(layout=fb.NCHW)) == 1 * 6 * 16 * 44 * 32 * 4
     assert fb.flashbev_workspace_bytes(good_params(layout=fb.NCHW, C=30)) == 0
+    # channels-last rows that are not whole 16-byte vectors: a copy with the rows padded to whole vectors
+    assert fb.flashbev_workspace_bytes(good_params(C=30)) == 1 * 6 * 16 * 44 * 32 * 4
+    assert fb.flashbev_workspace_bytes(good_params(C=33, feat_dtype=fb.BF16)) == 1 * 6 * 16 * 44 * 40 * 2
     # a workspace that is too small or misaligned is not used: forcing the tiled kernel is refused on the host
     for ws, nbytes in ((8192, 100), (8200, 1 << 30)):
         p = good_params(layout=fb.NCHW, kernel=fb.KERNEL_TILED)

@@ -86,9 +86,13 @@ def test_channel_counts_general_pose(oracle, reduce, kernel, dtype, C):
 
 
 @pytest.mark.parametrize("dtype,C", [("f32", 3), ("f32", 1), ("f32", 7), ("bf16", 5), ("bf16", 12)])
-def test_channel_counts_without_16_byte_rows_use_the_generic_kernel(oracle, dtype, C):
+def test_channel_counts_without_16_byte_rows(oracle, dtype, C):
+    """With the scratch the torch wrapper lends: the tiled kernel on a zero-padded copy; the generic kernel when asked
+    for; and the tiled kernel forced on the caller's own rows is refused on the host."""
     inp = small(40 + C, C=C, dtype=dtype)
     _, _, kname = check_small(oracle, inp, EQ1)
+    assert kname.startswith("tiled") and kname.endswith("padded")
+    _, _, kname = check_small(oracle, inp, EQ1, fb.KERNEL_PER_OUTPUT)
     assert kname.startswith("per_output") and kname.endswith("x1")
     w = inp.workload
     p = fb.make_params(16, fb.F32 if dtype == "f32" else fb.BF16, 16, w.B, w.N, C, w.feat_hw, w.img_hw, w.bev_range,

@@ -131,3 +131,29 @@ def test_feature_pointer_aligned_to_16_but_not_32_bytes(name):
     a = fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, w.reduce)
     b = fb.sampling_vt(shifted, m, w.img_hw, w.bev_range, w.grid, w.reduce)
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("reduce", [SUM, MEAN, EQ1])
+@pytest.mark.parametrize("dtype,C", [("f32", 1), ("f32", 5), ("f32", 82), ("bf16", 7), ("bf16", 12), ("bf16", 130)])
+def test_ragged_channel_counts_on_the_tiled_kernel(oracle, reduce, dtype, C):
+    """Channels-last rows that are not whole 16-byte vectors: with the scratch lent the tiled kernel runs on a copy with
+    zero-padded rows and writes the caller's ragged rows one channel at a time; without it the generic kernel runs.
+    Same oracle either way, and not a byte outside the output rows is touched."""
+    import torch
+    w = wl.Workload(f"ragged{C}", 3300 + C, 2, 5, C, dtype, (10, 14), (80, 112), (17, 13, 6),
+                    (-10.0, 10.0, -10.0, 10.0, -3.0, 2.0), 0, general_pose=True)
+    inp = wl.make_inputs(w)
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, reduce)
+    f, m = _cuda_features(inp, fb.NHWC)
+    X, Y, Z = w.grid
+    for workspace in (True, False):
+        cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=f.device)
+        guard = torch.full((w.B * X * Y * C + 64,), 7.0, device=f.device)
+        out = guard[:w.B * X * Y * C].view(w.B, X, Y, C)
+        fb.sampling_vt(f, m, w.img_hw, w.bev_range, w.grid, reduce, out=out, valid_count=cnt, workspace=workspace)
+        name = fb.flashbev_last_kernel_name()
+        assert name == (("tiled_bf16_padded" if dtype == "bf16" else "tiled_f32_padded") if workspace else
+                        ("per_output_bf16x1" if dtype == "bf16" else "per_output_f32x1"))
+        assert fb.flashbev_last_launch_count() == (2 if workspace else 1)
+        assert bool((guard[w.B * X * Y * C:] == 7.0).all())
+        parity.assert_parity(w, ref, out.cpu().numpy(), cnt.cpu().numpy(), f"[ragged {name}]", check_fraction=False)

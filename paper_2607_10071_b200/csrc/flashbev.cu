@@ -102,9 +102,19 @@ __device__ __forceinline__ int fb_idx(long long i, long long n, unsigned *err)
     }
     return (int)i;
 }
+__device__ __forceinline__ size_t fb_idx64(size_t i, size_t n, unsigned *err)
+{
+    if (i >= n) {
+        if (err) atomicAdd(err, 1u);
+        return 0;
+    }
+    return i;
+}
 #define FB_IDX(i, n, err) fb_idx((long long)(i), (long long)(n), (err))
+#define FB_IDX64(i, n, err) fb_idx64((size_t)(i), (size_t)(n), (err))
 #else
 #define FB_IDX(i, n, err) (i)
+#define FB_IDX64(i, n, err) (i)
 #endif
 
 struct Sample {

@@ -944,7 +944,7 @@ __global__ void __launch_bounds__(WARPS * 32, (V == 4 ? 12 : FB_WARPS_PER_SM) / 
                                     for (int hl = 0; hl < 2; ++hl) {
                                         const int ch = out_lane + v * vstride + e * 2 + hl;
                                         if (ch >= p.out_c) continue;  // (padding channels of the copy)
-                                        const size_t idx = at + (size_t)ch * p.out_chs;
+                                        const size_t idx = FB_IDX64(at + (size_t)ch * p.out_chs, (size_t)p.B * p.out_bs, p.err);
                                         float val = hl ? acc[v][e].y : acc[v][e].x;
                                         if (p.out_bf16) {
                                             uint16_t *ob = reinterpret_cast<uint16_t *>(p.out) + idx;

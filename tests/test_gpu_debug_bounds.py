@@ -156,3 +156,40 @@ def test_random_problems_and_hints_make_no_out_of_range_index(oracle, checked, c
     assert violations == 0, f"{case}: {violations} out-of-range indices"
     ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, case["reduce"])
     parity.assert_parity(w, ref, out, cnt, f"[checked build {case}]", check_fraction=False, large_outputs=True)
+
+
+@pytest.mark.parametrize("layout,dtype,C", [(fb.NCHW, "f32", 32), (fb.NCHW, "bf16", 72), (fb.NHWC, "f32", 82), (fb.NHWC, "bf16", 13)])
+def test_copies_in_a_lent_workspace_make_no_out_of_range_index(oracle, checked, layout, dtype, C):
+    """Planar tensors and ragged channel counts in the checked build: transposed / padded copy in the workspace, scalar
+    stores with the caller's strides -- no index out of range, nothing written past the output, the oracle's numbers."""
+    import torch
+    w = wl.Workload("lent", 8800 + C, 2, 5, C, dtype, (10, 14), (80, 112), (23, 17, 12),
+                    (-10.0, 10.0, -10.0, 10.0, -3.0, 2.0), 2, general_pose=False, yaw_jitter_deg=3.0)
+    inp = wl.make_inputs(w)
+    dev = torch.device("cuda:0")
+    if dtype == "bf16":
+        f = torch.from_numpy(inp.features_bf16.view(np.int16)).to(dev).view(torch.bfloat16)
+    else:
+        f = torch.from_numpy(inp.features).to(dev)
+    if layout == fb.NCHW:
+        f = f.permute(0, 1, 4, 2, 3).contiguous()
+    m = torch.from_numpy(inp.lidar2img).to(dev)
+    X, Y, Z = w.grid
+    n_out = w.B * X * Y * C
+    guard = torch.full((n_out + 64,), 7.0, device=dev)
+    cnt = torch.full((w.B, X, Y), -1, dtype=torch.int32, device=dev)
+    word = torch.zeros(1, dtype=torch.int32, device=dev)
+    p = fb.make_params(f.data_ptr(), fb.BF16 if dtype == "bf16" else fb.F32, m.data_ptr(), w.B, w.N, C, w.feat_hw, w.img_hw,
+                       w.bev_range, w.grid, 2, guard.data_ptr(), cnt.data_ptr(), layout=layout, debug_error_word=word.data_ptr())
+    need = fb.flashbev_workspace_bytes(p)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    p.workspace, p.workspace_bytes = ws.data_ptr(), need
+    fb.flashbev_sampling_vt(p, torch.cuda.current_stream().cuda_stream, library=checked)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    assert bool((guard[n_out:] == 7.0).all())
+    out = guard[:n_out].view((w.B, C, X, Y) if layout == fb.NCHW else (w.B, X, Y, C))
+    out = out.permute(0, 2, 3, 1) if layout == fb.NCHW else out
+    ref = oracle.sampling_vt(inp.features, inp.lidar2img, w.img_hw, w.bev_range, w.grid, 2)
+    parity.assert_parity(w, ref, out.cpu().numpy(), cnt.cpu().numpy(), "[lent workspace, checked build]", check_fraction=False)

@@ -424,6 +424,15 @@ def sampling_vt_multires(features, lidar2img, img_hw, bev_range, grid, reduce=RE
     base = make_params(f0.data_ptr(), dt, lidar2img.data_ptr(), B, N, C, hws[0], img_hw, bev_range, (X, Y, Z),
                        reduce, out.data_ptr(), None if valid_count is None else valid_count.data_ptr(),
                        kernel, tune, layout, F32)
+    # planar tensors and ragged channel counts: lend the scratch of the largest level (the levels run one after another)
+    need = 0
+    for f, hw in zip(features, hws):
+        base.features, base.feat_h, base.feat_w = f.data_ptr(), hw[0], hw[1]
+        need = max(need, flashbev_workspace_bytes(base))
+    base.features, base.feat_h, base.feat_w = f0.data_ptr(), hws[0][0], hws[0][1]
+    if need:
+        ws = torch.empty(need, dtype=torch.uint8, device=f0.device)
+        base.workspace, base.workspace_bytes = ws.data_ptr(), need
     if stream is None:
         stream = torch.cuda.current_stream(f0.device).cuda_stream
     with torch.cuda.device(f0.device):

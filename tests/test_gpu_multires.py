@@ -57,17 +57,25 @@ def test_pyramid_parity(oracle, name, levels, reduce):
     print(name, levels, reduce, rep)
 
 
-@pytest.mark.parametrize("kernel,layout", [(fb.KERNEL_PER_OUTPUT, fb.NHWC), (fb.KERNEL_AUTO, fb.NCHW)])
+@pytest.mark.parametrize("kernel,layout", [(fb.KERNEL_PER_OUTPUT, fb.NHWC), (fb.KERNEL_PER_OUTPUT, fb.NCHW),
+                                           (fb.KERNEL_AUTO, fb.NCHW), (fb.KERNEL_AUTO, fb.NHWC)])
 @pytest.mark.parametrize("dtype,C", [("f32", 6), ("bf16", 24)])
-def test_pyramid_generic_kernels(oracle, kernel, layout, dtype, C):
-    """Per-output kernels (odd channel counts, planar tensors) add the levels the same way."""
+def test_pyramid_generic_kernels_and_lent_workspace(oracle, kernel, layout, dtype, C):
+    """Per-output kernels (odd channel counts, planar tensors) add the levels the same way, and so do the tiled kernel's
+    scalar-store instances on the copies in the workspace the wrapper lends (planar tensors, ragged channel counts)."""
     w = wl.Workload(f"mrg{C}", 5100 + C, 2, 5, C, dtype, (11, 15), (88, 120), (13, 11, 6),
                     (-10.0, 10.0, -10.0, 10.0, -3.0, 2.0), 0, general_pose=True)
     feats, bits, mats = wl.make_pyramid_inputs(w, 3)
     ref = oracle.sampling_vt_multires(feats, mats, w.img_hw, w.bev_range, w.grid, EQ1)
     f, m = _upload(w, feats, bits, mats, layout)
     out = fb.sampling_vt_multires(f, m, w.img_hw, w.bev_range, w.grid, EQ1, kernel=kernel, layout=layout)
-    assert fb.flashbev_last_kernel_name().startswith("per_output")
+    whole = (C * (4 if dtype == "f32" else 2)) % 16 == 0
+    if kernel == fb.KERNEL_PER_OUTPUT or (layout == fb.NCHW and not whole):
+        assert fb.flashbev_last_kernel_name().startswith("per_output")
+    elif layout == fb.NCHW:
+        assert fb.flashbev_last_kernel_name().endswith("nchw")
+    else:
+        assert fb.flashbev_last_kernel_name().endswith("padded" if not whole else "v1")
     o = out.permute(0, 2, 3, 1) if layout == fb.NCHW else out
     parity.assert_parity(w, ref, o.cpu().numpy(), None, "[multires generic]", check_fraction=False)
 

@@ -296,6 +296,31 @@ def test_host_buffer_entry_point_with_planar_tensors(oracle, bench_inputs):
     assert float((full - hout).abs().max()) <= 1e-5
 
 
+def test_host_buffer_entry_point_with_ragged_channel_counts(oracle):
+    """Host tensors with C = 30 fp32 (120-byte rows): the staging area has room for the padded copy, so the tiled kernel
+    runs; cut down to its compulsory part the generic kernel runs."""
+    import torch
+    w = wl.get("tiny", C=30)
+    inp = wl.make_inputs(w)
+    X, Y, Z = w.grid
+    hf = torch.from_numpy(inp.features).pin_memory()
+    hm = torch.from_numpy(inp.lidar2img).pin_memory()
+    ref = oracle_of(oracle, inp, w.reduce)
+    for cut in (False, True):
+        hout = torch.full((w.B, X, Y, w.C), float("nan")).pin_memory()
+        hcnt = torch.full((w.B, X, Y), -1, dtype=torch.int32).pin_memory()
+        p = fb.make_params(hf.data_ptr(), fb.F32, hm.data_ptr(), w.B, w.N, w.C, w.feat_hw, w.img_hw, w.bev_range, w.grid,
+                           w.reduce, hout.data_ptr(), hcnt.data_ptr())
+        need, ws = fb.flashbev_host_staging_bytes(p), fb.flashbev_workspace_bytes(p)
+        assert ws == inp.features.nbytes // 30 * 32
+        staging = torch.empty(need, dtype=torch.uint8, device="cuda:0")
+        s = torch.cuda.Stream()
+        fb.flashbev_sampling_vt_host(p, staging.data_ptr(), need - ws if cut else need, s.cuda_stream)
+        s.synchronize()
+        assert fb.flashbev_last_kernel_name() == ("per_output_f32x1" if cut else "tiled_f32_padded")
+        parity.assert_parity(w, ref, hout.numpy(), hcnt.numpy(), "[host entry, ragged]")
+
+
 def test_runs_on_a_caller_stream(oracle, bench_inputs):
     import torch
     inp = bench_inputs["tiny"]

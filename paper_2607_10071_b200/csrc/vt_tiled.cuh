@@ -642,8 +642,10 @@ __device__ __forceinline__ int build_columns(const KParams &p, WarpCtx cx, int j
         int mine = 0;  // records of this lane's column
         if (j < ncols) {
             sm.colw[j] = wbase;
+            // runs of equal length (17 rows: 9 + 8, not 16 + 1): the walkers of a round finish together
+            const int per = runs > 1 ? (units + runs - 1) / runs : units;
             for (int i = 0; i < runs; ++i) {
-                const int u0 = i * p.walk, len = min(p.walk, units - u0);
+                const int u0 = i * per, len = min(per, units - u0);
                 sm.wk[FB_IDX(wbase + i, p.wcap, p.err)] = (uint32_t)j | ((uint32_t)u0 << 8) | ((uint32_t)(len - 1) << 24);
                 sm.woff[FB_IDX(wbase + i, p.wcap + 1, p.err)] = mine;
                 mine += affine ? affine_run_records(D, len) : walk_general<false>(p, sm, cx.mats, D, u0, len, nullptr, nullptr, 0);

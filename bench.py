@@ -40,7 +40,7 @@ MIN_LAUNCHES_PER_STEP = 64
 # launches taken from the middle of a step of rotating frames -- the regime that is timed -- summarised under
 # profiles/vt_tiled_kernel_<workload>.md.  The output of a launch is still partly in the 126 MB L2 when its kernel
 # ends, so these figures can lie below the algorithmic bytes: see `traffic_note` in the JSON line.
-NCU_DRAM_TRAFFIC = {"tiny": 0.342e6, "representative": 4.78e6, "half_taller": 8.20e6, "long_range": 41.00e6, "high_res": 21.64e6}
+NCU_DRAM_TRAFFIC = {"tiny": 0.342e6, "representative": 4.78e6, "half_taller": 8.20e6, "long_range": 41.00e6, "high_res": 21.45e6}
 TRAFFIC_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum of one launch captured in the middle of a rotating-frame "
                 "step (ncu, one pass); part of a launch's output is written back from L2 after its kernel ends, so the "
                 "figure can be below the algorithmic bytes")

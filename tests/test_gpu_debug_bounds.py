@@ -135,7 +135,7 @@ def checked_cases(draw):
         tail=draw(st.integers(0, 7)), order=draw(st.sampled_from([0, 1 << 28, 1 << 18, 3 << 18])))
 
 
-@settings(max_examples=50, deadline=None, derandomize=True,
+@settings(max_examples=150, deadline=None, derandomize=True,
           suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
 @given(case=checked_cases())
 def test_random_problems_and_hints_make_no_out_of_range_index(oracle, checked, case):

@@ -25,7 +25,7 @@ def cases(draw):
         walk=draw(st.sampled_from([0, 1, 3, 8])))
 
 
-@settings(max_examples=60, deadline=None, derandomize=True,
+@settings(max_examples=200, deadline=None, derandomize=True,
           suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
 @given(case=cases())
 def test_random_small_problems_match_the_oracle(oracle, case):

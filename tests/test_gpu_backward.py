@@ -6,6 +6,7 @@ collects up to a few thousand fp32 contributions; their rounding errors add like
 """
 import numpy as np
 import pytest
+from hypothesis import HealthCheck, given, settings, strategies as st
 
 from paper_2607_10071_b200 import binding as fb
 from paper_2607_10071_b200 import workloads as wl
@@ -103,3 +104,34 @@ def test_backward_rejects_what_it_does_not_support():
                          (dict(grid=(0, 50, 4)), fb.INVALID_ARG)):
         p = fb.make_backward_params(**{**good, **over})
         assert fb.flashbev_sampling_vt_backward(p, None, check=False) == status, over
+
+
+@st.composite
+def backward_cases(draw):
+    return dict(
+        seed=draw(st.integers(0, 10_000)), C=4 * draw(st.sampled_from([1, 2, 3, 5, 8, 10, 16, 20, 33])),
+        B=draw(st.integers(1, 2)), N=draw(st.integers(1, 7)),
+        feat=(draw(st.integers(1, 16)), draw(st.integers(1, 20))),
+        grid=(draw(st.integers(1, 21)), draw(st.integers(1, 21)), draw(st.sampled_from([1, 2, 5, 8, 16, 40, 97]))),
+        general=draw(st.booleans()), rng_xy=draw(st.sampled_from([3.0, 10.0, 40.0])),
+        reduce=draw(st.sampled_from([SUM, MEAN, EQ1])),
+        walk=draw(st.sampled_from([0, 1, 4, 32])), slots=draw(st.sampled_from([0, 64, 128, 1024])),
+        shape=draw(st.sampled_from([0, (1 << 4) | (1 << 8), (2 << 4) | (2 << 8), (4 << 4) | (2 << 8)])))
+
+
+@settings(max_examples=80, deadline=None, derandomize=True,
+          suppress_health_check=[HealthCheck.function_scoped_fixture, HealthCheck.too_slow])
+@given(case=backward_cases())
+def test_backward_random_problems_match_the_oracle(oracle, case):
+    """Random rigs (surround and general pose), shapes, reduce modes and launch-geometry hints against the oracle's
+    backward; hints the kernel cannot be configured for are refused on the host."""
+    w = wl.Workload("bwd_prop", 7000 + case["seed"], case["B"], case["N"], case["C"], "f32", case["feat"],
+                    (case["feat"][0] * 8, case["feat"][1] * 8), case["grid"],
+                    (-case["rng_xy"], case["rng_xy"], -case["rng_xy"], case["rng_xy"], -3.0, 2.5), case["reduce"],
+                    general_pose=case["general"], yaw_jitter_deg=5.0)
+    inp = wl.make_inputs(w)
+    tune = (0, 0, case["walk"], case["shape"] | ((case["slots"] // 16) << 20))
+    try:
+        check(oracle, w, inp.lidar2img, case["reduce"], seed=case["seed"], tune=tune)
+    except fb.FlashBevError as e:
+        assert e.status == fb.UNSUPPORTED, e
